@@ -1,0 +1,143 @@
+"""ctypes binding of the fp64 CPU oracle (`sr_ref.cpp`).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's cpu_baseline / reference legs.  The CUDA package never imports it.
+Arrays are numpy, outputs are float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sr_ref.cpp")
+_LIB = os.path.join(_HERE, "libsr_ref.so")
+
+F32, F16 = 0, 1
+CLAMP01, IDX_GLOBAL, COEF_COMPACT = 1, 2, 4
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ -O2 (plus OpenMP for the row loop) into libsr_ref.so."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        vp, i32, i64, u32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint
+        L.sr_ref_bicubic_upsample.argtypes = [vp, vp] + [i32] * 6
+        L.sr_ref_dict_regress_dense.argtypes = [vp, vp, i32, vp, vp] + [i32] * 7 + [u32, i32]
+        L.sr_ref_dict_select.argtypes = [vp, i32, vp, vp] + [i32] * 6
+        L.sr_ref_dict_regress_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp] + [i32] * 8 + [u32, i32]
+        L.sr_ref_regress_at.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, i64, vp] + [i32] * 8 + [u32, i32]
+        L.sr_ref_dict_select_at.argtypes = [vp, i32, vp, i64, vp] + [i32] * 6
+        L.sr_ref_max_threads.argtypes = []
+        for f in (L.sr_ref_bicubic_upsample, L.sr_ref_dict_regress_dense, L.sr_ref_dict_select,
+                  L.sr_ref_dict_regress_selected, L.sr_ref_regress_at, L.sr_ref_dict_select_at, L.sr_ref_max_threads):
+            f.restype = i32
+        _lib = L
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().sr_ref_max_threads())
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.float16:
+        return F16
+    raise TypeError(f"coefficients must be float32 or float16, got {a.dtype}")
+
+
+def _c(a, dt=None):
+    a = np.ascontiguousarray(a) if dt is None else np.ascontiguousarray(a, dtype=dt)
+    return a
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise ValueError(f"{what}: oracle status {status}")
+
+
+def bicubic_upsample(lr: np.ndarray, scale: int, threads: int = 0) -> np.ndarray:
+    lr = _c(lr, np.float32)
+    n, c, h, w = lr.shape
+    out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_bicubic_upsample(lr.ctypes.data, out.ctypes.data, n, c, h, w, scale, threads), "bicubic")
+    return out
+
+
+def dict_regress_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, threads: int = 0) -> np.ndarray:
+    lr, coef, dict_ = _c(lr, np.float32), _c(coef), _c(dict_, np.float32)
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    assert dict_.shape == (D, k * k) and coef.shape == (n, D, h * scale, w * scale), (dict_.shape, coef.shape)
+    out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_dict_regress_dense(lr.ctypes.data, coef.ctypes.data, _dtype_code(coef), dict_.ctypes.data,
+                                             out.ctypes.data, n, c, h, w, scale, k, D, flags, threads), "dense")
+    return out
+
+
+def dict_select(coef, s: int, want_sel: bool = False, threads: int = 0):
+    coef = _c(coef)
+    n, D, H, W = coef.shape
+    idx = np.empty((n, s, H, W), dtype=np.uint8)
+    sel = np.empty((n, s, H, W), dtype=np.float64) if want_sel else None
+    _check(_load().sr_ref_dict_select(coef.ctypes.data, _dtype_code(coef), idx.ctypes.data,
+                                      sel.ctypes.data if want_sel else None, n, H, W, D, s, threads), "select")
+    return (idx, sel) if want_sel else idx
+
+
+def dict_regress_selected(lr, coef_or_sel, idx, gamma, dict_, scale: int, k: int, s: int, flags: int = 0,
+                          threads: int = 0) -> np.ndarray:
+    lr, coef_or_sel, dict_ = _c(lr, np.float32), _c(coef_or_sel), _c(dict_, np.float32)
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    idx = None if idx is None else _c(idx, np.uint8)
+    gamma = None if gamma is None else _c(gamma, np.float32)
+    out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_dict_regress_selected(
+        lr.ctypes.data, coef_or_sel.ctypes.data, _dtype_code(coef_or_sel), None if idx is None else idx.ctypes.data,
+        None if gamma is None else gamma.ctypes.data, dict_.ctypes.data, out.ctypes.data, n, c, h, w, scale, k, D, s,
+        flags, threads), "selected")
+    return out
+
+
+def regress_at(mode: str, lr, coef_or_sel, idx, gamma, dict_, samples, scale: int, k: int, s: int = 0, flags: int = 0,
+               threads: int = 0) -> np.ndarray:
+    """Dense (`mode="dense"`) or selected regression at sampled flat [n][H][W] indices -> [nsamples][c]."""
+    lr, coef_or_sel, dict_ = _c(lr, np.float32), _c(coef_or_sel), _c(dict_, np.float32)
+    samples = _c(samples, np.int64)
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    idx = None if idx is None else _c(idx, np.uint8)
+    gamma = None if gamma is None else _c(gamma, np.float32)
+    out = np.empty((samples.size, c), dtype=np.float64)
+    _check(_load().sr_ref_regress_at(
+        0 if mode == "dense" else 1, lr.ctypes.data, coef_or_sel.ctypes.data, _dtype_code(coef_or_sel),
+        None if idx is None else idx.ctypes.data, None if gamma is None else gamma.ctypes.data, dict_.ctypes.data,
+        samples.ctypes.data, samples.size, out.ctypes.data, n, c, h, w, scale, k, D, s if s else D, flags, threads),
+        "regress_at")
+    return out
+
+
+def dict_select_at(coef, samples, s: int, threads: int = 0) -> np.ndarray:
+    coef = _c(coef)
+    samples = _c(samples, np.int64)
+    n, D, H, W = coef.shape
+    out = np.empty((samples.size, s), dtype=np.uint8)
+    _check(_load().sr_ref_dict_select_at(coef.ctypes.data, _dtype_code(coef), samples.ctypes.data, samples.size,
+                                         out.ctypes.data, n, H, W, D, s, threads), "select_at")
+    return out
