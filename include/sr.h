@@ -1,0 +1,132 @@
+/*
+ * sr.h - C ABI of the B200 (sm_100a) pixel-adaptive dictionary regression library.
+ *
+ * The library computes the last two stages of a LAPAR-style super-resolution
+ * model together with the up-sampling they consume (paper Section II-A,
+ * Eq. 2-3): the LR image is up-sampled to U, the k x k patch B_i of U around
+ * every HR pixel i is taken, the per-pixel filter F_i = Phi_i D is assembled
+ * from the dictionary D (L atoms of k*k taps; L is called D in `sr_dims`) and
+ * the pixel's coefficients Phi_i, and y_i = F_i B_i^T.  The filter matrix F and
+ * the patch matrix B never reach global memory.
+ *
+ * Conventions shared by every call
+ *   - Every data pointer is a DEVICE pointer; `stream` is a cudaStream_t passed
+ *     as void* (NULL = the legacy default stream).  `d` is a HOST pointer.
+ *   - Layouts, all contiguous, row-major, innermost index last:
+ *       lr        [n][c][h][w]           fp32   LR image
+ *       hr / out  [n][c][H][W]           fp32   H = h*scale, W = w*scale
+ *       coef      [n][D][H][W]           fp32 or binary16 (SR_F32 / SR_F16); one set per
+ *                                        frame, shared by the c channels
+ *       dict      [D][k*k]               fp32, tap j = a*k + b (a = row) multiplies
+ *                                        U[Y + a - p][X + b - p], p = (k-1)/2 (no flip)
+ *       idx       [n][s][H][W]           uint8, rank order (plane 0 = largest magnitude);
+ *                                        with SR_IDX_GLOBAL: idx[s]
+ *       sel       [n][s][H][W]           coefficient dtype; plane q = coefficient of idx plane q
+ *       gamma     [s]                    fp32 (SR_IDX_GLOBAL only)
+ *   - Ownership: the caller owns every buffer.  The library allocates nothing
+ *     the caller must free and keeps no reference after the call's work has
+ *     run.  Calls are asynchronous on `stream` and never synchronise the host;
+ *     buffers must stay valid until the stream reaches the kernels.  `out`
+ *     must not alias an input.
+ *   - Errors: every call returns an sr status.  Validation failures return
+ *     before anything is launched and write nothing.  Nothing throws, aborts or
+ *     prints.  A device-side wait that ran out of its iteration limit is
+ *     reported by sr_device_status (the output of that call is then undefined).
+ *   - Alignment: lr, hr/out, dict and gamma 4 bytes; coef/sel their element size
+ *     (the tensor-core path additionally needs coef 16-byte aligned and W a
+ *     multiple of 8; other inputs take the general path).
+ */
+#ifndef SR_H_
+#define SR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sr_dims {
+    int32_t n, c, h, w; /* LR batch, channels, height, width (each >= 1)                 */
+    int32_t scale;      /* integer up-scaling factor r in [1, 8]                          */
+    int32_t k;          /* atom / patch side, odd, in {1,3,5,7,9}                         */
+    int32_t D;          /* number of dictionary atoms (the paper's L), 1..256             */
+} sr_dims;
+
+enum { SR_F32 = 0, SR_F16 = 1 }; /* coefficient storage type */
+
+enum {
+    SR_CLAMP01 = 1u,      /* clamp the output to [0,1] as the last step                                */
+    SR_IDX_GLOBAL = 2u,   /* idx[s] (+ gamma[s]) is one atom subset for every pixel                    */
+    SR_COEF_COMPACT = 4u  /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
+};
+
+enum {
+    SR_OK = 0,
+    SR_ERR_NULL = 1,        /* a required pointer is NULL                        */
+    SR_ERR_SHAPE = 2,       /* a size is out of range (n,c,h,w,D < 1; s < 1 or s > D; total size overflow) */
+    SR_ERR_UNSUPPORTED = 3, /* scale not in [1,8]; k even or > 9; D > 256; unknown dtype or flag */
+    SR_ERR_ALIGN = 4,       /* a pointer is not aligned to its element size      */
+    SR_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed              */
+    SR_ERR_TIMEOUT = 6      /* device status only: a bounded device-side wait expired */
+};
+
+/*
+ * Stage 1 alone (Section II-A, "the LR input is up-sampled"): hr = bicubic(lr).
+ * Keys cubic convolution with a = -0.75, half-pixel centres
+ * (src = (X + 1/2)/scale - 1/2), tap indices clamped to the image; the result
+ * is not clamped.  d->k and d->D are ignored.
+ */
+int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream);
+
+/*
+ * Stages 1, 3 and 4 with every atom (Eq. 2: y_i = F_i B_i^T with F_i = Phi_i D;
+ * image form Eq. 3): out[n][c][Y][X] = sum_j (sum_l coef[n][l][Y][X] * dict[l][j]) * B_c[j],
+ * patch positions clamped to the HR image (edge replicate).  fp32 accumulation.
+ * flags: SR_CLAMP01 or 0.
+ */
+int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out,
+                          const sr_dims* d, uint32_t flags, void* stream);
+
+/*
+ * Per-pixel top-s selection (the dictionary selective strategy applied per HR
+ * pixel; the paper's Section III-A selects one subset for the whole model,
+ * which is the SR_IDX_GLOBAL mode of sr_dict_regress_selected): for every
+ * pixel the s atoms with the largest |coef|, ties to the lower atom index,
+ * written in rank order.  The ordering key is the coefficient's bit pattern
+ * with the sign cleared, so -0/+0 and +x/-x tie.  `sel` may be NULL; otherwise
+ * it receives the selected coefficients.  flags must be 0.  d->c, d->k unused.
+ */
+int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, const sr_dims* d, int s,
+                   uint32_t flags, void* stream);
+
+/*
+ * Stages 1, 3 and 4 with s atoms per pixel (Section II-A: computations the
+ * dictionary gates are skipped; Section III-A, Eq. 6 and Eq. 9 for the global
+ * form): out = sum_j (sum_q w_q * dict[a_q][j]) * B_c[j].
+ *   flags = 0:               a_q = idx[n][q][Y][X], w_q = coef[n][a_q][Y][X]
+ *                            (idx == NULL: the top-s atoms are chosen inside the call and never stored)
+ *   SR_COEF_COMPACT:         w_q = coef_or_sel[n][q][Y][X]  (idx required)
+ *   SR_IDX_GLOBAL:           a_q = idx[q], w_q = gamma[q] * coef[n][a_q][Y][X]  (gamma NULL = 1);
+ *                            with SR_COEF_COMPACT, w_q = gamma[q] * coef_or_sel[n][q][Y][X]
+ * Kept coefficients are used unchanged (no renormalisation).  An idx value >= D
+ * is the caller's error: that pixel's value is then undefined, but no
+ * out-of-range access is made (the value is clamped to D-1).
+ */
+int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_dtype, const uint8_t* idx,
+                             const float* gamma, const float* dict, float* out, const sr_dims* d, int s,
+                             uint32_t flags, void* stream);
+
+/* Text for a status code (static storage, never NULL). */
+const char* sr_status_string(int status);
+
+/*
+ * Synchronises `stream`, then reads and clears the device status word of the
+ * current device into *out_status (SR_OK or SR_ERR_TIMEOUT).  Returns SR_OK,
+ * SR_ERR_NULL or SR_ERR_CUDA.
+ */
+int sr_device_status(void* stream, int* out_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SR_H_ */

@@ -1,0 +1,165 @@
+"""Thin Python binding of the C-ABI library (argument marshalling only).
+
+Every function takes torch CUDA tensors (used purely as device memory), checks their dtype, shape and
+contiguity, and passes raw pointers, the problem dimensions and the current CUDA stream to the
+library entry point of the same name. Nothing is computed in Python and nothing falls back to the CPU:
+if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsr.so")
+
+SR_F32, SR_F16 = 0, 1
+SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT = 1, 2, 4
+SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
+
+EXPORTS = ("sr_bicubic_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
+           "sr_status_string", "sr_device_status")
+
+
+class sr_dims(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int32) for name in ("n", "c", "h", "w", "scale", "k", "D")]
+
+
+class SrError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libsr.so; raises if it has not been built (there is no other implementation to fall back to)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2303_08999_b200.build`")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, u32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint32
+        dp = ctypes.POINTER(sr_dims)
+        lib.sr_bicubic_upsample.argtypes = [vp, vp, dp, vp]
+        lib.sr_dict_regress_dense.argtypes = [vp, vp, i32, vp, vp, dp, u32, vp]
+        lib.sr_dict_select.argtypes = [vp, i32, vp, vp, dp, i32, u32, vp]
+        lib.sr_dict_regress_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp, dp, i32, u32, vp]
+        lib.sr_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+        for name in EXPORTS:
+            getattr(lib, name).restype = i32
+        lib.sr_status_string.argtypes = [i32]
+        lib.sr_status_string.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().sr_status_string(status).decode()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _dev(t: torch.Tensor, dtype, what: str) -> torch.Tensor:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{what} must be a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def _coef_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return SR_F16
+    if t.dtype == torch.float32:
+        return SR_F32
+    raise TypeError("coefficients must be float16 or float32")
+
+
+def _check(status: int, what: str):
+    if status != SR_OK:
+        raise SrError(status, what)
+
+
+def sr_bicubic_upsample(lr: torch.Tensor, scale: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    lr = _dev(lr, torch.float32, "lr")
+    n, c, h, w = lr.shape
+    if out is None:
+        out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float32, device=lr.device)
+    _dev(out, torch.float32, "out")
+    assert out.shape == (n, c, h * scale, w * scale)
+    d = sr_dims(n, c, h, w, scale, 1, 1)
+    _check(load_library().sr_bicubic_upsample(_ptr(lr), _ptr(out), ctypes.byref(d), _stream()), "sr_bicubic_upsample")
+    return out
+
+
+def sr_dict_regress_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, out=None) -> torch.Tensor:
+    lr, dict_ = _dev(lr, torch.float32, "lr"), _dev(dict_, torch.float32, "dict")
+    code = _coef_code(coef)
+    _dev(coef, coef.dtype, "coef")
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    assert dict_.shape == (D, k * k) and coef.shape == (n, D, h * scale, w * scale)
+    if out is None:
+        out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float32, device=lr.device)
+    _dev(out, torch.float32, "out")
+    d = sr_dims(n, c, h, w, scale, k, D)
+    _check(load_library().sr_dict_regress_dense(_ptr(lr), _ptr(coef), code, _ptr(dict_), _ptr(out), ctypes.byref(d),
+                                                flags, _stream()), "sr_dict_regress_dense")
+    return out
+
+
+def sr_dict_select(coef, s: int, want_sel: bool = False, idx=None, sel=None):
+    code = _coef_code(coef)
+    _dev(coef, coef.dtype, "coef")
+    n, D, H, W = coef.shape
+    if idx is None:
+        idx = torch.empty((n, s, H, W), dtype=torch.uint8, device=coef.device)
+    _dev(idx, torch.uint8, "idx")
+    if want_sel and sel is None:
+        sel = torch.empty((n, s, H, W), dtype=coef.dtype, device=coef.device)
+    if sel is not None:
+        _dev(sel, coef.dtype, "sel")
+    d = sr_dims(n, 1, H, W, 1, 1, D)
+    _check(load_library().sr_dict_select(_ptr(coef), code, _ptr(idx), _ptr(sel), ctypes.byref(d), s, 0, _stream()),
+           "sr_dict_select")
+    return (idx, sel) if sel is not None else idx
+
+
+def sr_dict_regress_selected(lr, coef_or_sel, idx, gamma, dict_, scale: int, k: int, s: int, flags: int = 0,
+                             out=None) -> torch.Tensor:
+    lr, dict_ = _dev(lr, torch.float32, "lr"), _dev(dict_, torch.float32, "dict")
+    code = _coef_code(coef_or_sel)
+    _dev(coef_or_sel, coef_or_sel.dtype, "coef_or_sel")
+    if idx is not None:
+        _dev(idx, torch.uint8, "idx")
+    if gamma is not None:
+        _dev(gamma, torch.float32, "gamma")
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    assert dict_.shape == (D, k * k)
+    planes = s if (flags & SR_COEF_COMPACT) else D
+    assert coef_or_sel.shape == (n, planes, h * scale, w * scale)
+    if out is None:
+        out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float32, device=lr.device)
+    _dev(out, torch.float32, "out")
+    d = sr_dims(n, c, h, w, scale, k, D)
+    _check(load_library().sr_dict_regress_selected(_ptr(lr), _ptr(coef_or_sel), code, _ptr(idx), _ptr(gamma),
+                                                   _ptr(dict_), _ptr(out), ctypes.byref(d), s, flags, _stream()),
+           "sr_dict_regress_selected")
+    return out
+
+
+def sr_device_status() -> int:
+    """Synchronises the current stream and returns (and clears) the device status word."""
+    v = ctypes.c_int(0)
+    _check(load_library().sr_device_status(_stream(), ctypes.byref(v)), "sr_device_status")
+    return v.value

@@ -1,0 +1,182 @@
+// C ABI entry points: argument validation, path selection, status reporting.
+#include <math.h>
+
+#include "sr_common.cuh"
+#include "sr_umma.cuh"
+
+namespace sr {
+
+__device__ int g_status_word = 0;
+
+int* device_status_word()
+{
+    // One lookup per device, cached (the symbol's address differs per device).
+    static int* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        cache[dev] = (int*)p;
+    }
+    return cache[dev];
+}
+
+// Keys cubic-convolution weights (a = -0.75) for every phase of an integer scale, computed in
+// double and rounded once. src = (X + 1/2)/r - 1/2 = (2X + 1 - r) / (2r) in exact integers.
+BicubicPhases make_phases(int r)
+{
+    BicubicPhases ph{};
+    const double A = -0.75;
+    for (int p = 0; p < r && p < kMaxScale; ++p) {
+        const int num = 2 * p + 1 - r;                     // numerator of src relative to q = X / r
+        const int fl = (num >= 0) ? num / (2 * r) : -((-num + 2 * r - 1) / (2 * r));
+        const double t = (double)(num - fl * 2 * r) / (double)(2 * r);
+        auto inner = [&](double z) { return ((A + 2.0) * z - (A + 3.0)) * z * z + 1.0; };
+        auto outer = [&](double z) { return ((A * z - 5.0 * A) * z + 8.0 * A) * z - 4.0 * A; };
+        ph.w[p][0] = (float)outer(t + 1.0);
+        ph.w[p][1] = (float)inner(t);
+        ph.w[p][2] = (float)inner(1.0 - t);
+        ph.w[p][3] = (float)outer(2.0 - t);
+        ph.base[p] = fl - 1;
+    }
+    return ph;
+}
+
+static int check_dims(const sr_dims* d, bool need_kD)
+{
+    if (!d) return SR_ERR_NULL;
+    if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return SR_ERR_SHAPE;
+    if (d->scale < 1 || d->scale > kMaxScale) return SR_ERR_UNSUPPORTED;
+    if (need_kD) {
+        if (d->D < 1) return SR_ERR_SHAPE;
+        if (d->D > 256) return SR_ERR_UNSUPPORTED;
+        if (d->k < 1 || d->k > kMaxK || (d->k % 2) == 0) return SR_ERR_UNSUPPORTED;
+    }
+    // keep every flat index inside int64 and every per-plane index inside int32
+    const int64_t H = (int64_t)d->h * d->scale, W = (int64_t)d->w * d->scale;
+    if (H * W > (int64_t)0x7FFFFFFF) return SR_ERR_SHAPE;
+    const int64_t planes = (int64_t)d->n * (need_kD ? (d->D > d->c ? d->D : d->c) : d->c);
+    if (planes > ((int64_t)1 << 40) / (H * W)) return SR_ERR_SHAPE;
+    return SR_OK;
+}
+
+static Problem make_problem(const sr_dims* d, int s, uint32_t flags)
+{
+    Problem pb{};
+    pb.n = d->n; pb.c = d->c; pb.h = d->h; pb.w = d->w; pb.r = d->scale; pb.k = d->k; pb.D = d->D;
+    pb.H = d->h * d->scale; pb.W = d->w * d->scale;
+    pb.s = s; pb.flags = flags;
+    pb.ph = make_phases(d->scale);
+    return pb;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+} // namespace sr
+
+using namespace sr;
+
+extern "C" {
+
+int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream)
+{
+    if (!lr || !hr || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, false)) return e;
+    if (!aligned(lr, 4) || !aligned(hr, 4)) return SR_ERR_ALIGN;
+    sr_dims dd = *d;
+    dd.k = 1; dd.D = 1;
+    const Problem pb = make_problem(&dd, 1, 0);
+    return launch_bicubic(lr, hr, pb, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out,
+                          const sr_dims* d, uint32_t flags, void* stream)
+{
+    if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)SR_CLAMP01) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
+        return SR_ERR_ALIGN;
+    const Problem pb = make_problem(d, d->D, flags);
+    cudaError_t err;
+    if (umma_supported(kModeDense, coef, coef_dtype, pb))
+        err = launch_regress_umma(kModeDense, lr, coef, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
+    else
+        err = launch_regress_fma(kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
+    return err == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, const sr_dims* d, int s, uint32_t flags,
+                   void* stream)
+{
+    if (!coef || !idx || !d) return SR_ERR_NULL;
+    sr_dims dd = *d;
+    dd.c = 1; dd.k = 1;
+    if (int e = check_dims(&dd, true)) return e;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags != 0) return SR_ERR_UNSUPPORTED;
+    if (s < 1 || s > d->D) return SR_ERR_SHAPE;
+    const size_t esz = coef_dtype == SR_F16 ? 2 : 4;
+    if (!aligned(coef, esz) || (sel && !aligned(sel, esz))) return SR_ERR_ALIGN;
+    const Problem pb = make_problem(&dd, s, 0);
+    return launch_select(coef, coef_dtype, idx, sel, pb, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_dtype, const uint8_t* idx,
+                             const float* gamma, const float* dict, float* out, const sr_dims* d, int s,
+                             uint32_t flags, void* stream)
+{
+    if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT)) return SR_ERR_UNSUPPORTED;
+    if (s < 1 || s > d->D) return SR_ERR_SHAPE;
+    if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
+    if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
+        !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
+        return SR_ERR_ALIGN;
+    const Problem pb = make_problem(d, s, flags);
+    int mode;
+    if (flags & SR_IDX_GLOBAL) mode = kModeGlobal;
+    else if (flags & SR_COEF_COMPACT) mode = kModeCompact;
+    else mode = idx ? kModeIdx : kModeFusedSelect;
+    cudaError_t err;
+    if (umma_supported(mode, coef_or_sel, coef_dtype, pb))
+        err = launch_regress_umma(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
+    else
+        err = launch_regress_fma(mode, lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, pb, (cudaStream_t)stream);
+    return err == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+const char* sr_status_string(int status)
+{
+    switch (status) {
+    case SR_OK: return "ok";
+    case SR_ERR_NULL: return "a required pointer is NULL";
+    case SR_ERR_SHAPE: return "a size is out of range";
+    case SR_ERR_UNSUPPORTED: return "unsupported scale, atom size, atom count, dtype or flag";
+    case SR_ERR_ALIGN: return "a pointer is misaligned";
+    case SR_ERR_CUDA: return "a CUDA call or kernel launch failed";
+    case SR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+    }
+}
+
+int sr_device_status(void* stream, int* out_status)
+{
+    if (!out_status) return SR_ERR_NULL;
+    int* word = device_status_word();
+    if (!word) return SR_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, word, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SR_ERR_CUDA;
+    if (cudaMemsetAsync(word, 0, sizeof(int), st) != cudaSuccess) return SR_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SR_ERR_CUDA;
+    *out_status = v;
+    return SR_OK;
+}
+
+} // extern "C"

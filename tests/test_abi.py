@@ -1,0 +1,89 @@
+"""The C-ABI library loads, exports every symbol the public header declares, and validates arguments
+on the host before anything is launched (so these calls need no GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2303_08999_b200 as sr
+from paper_2303_08999_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return sr.load_library()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "sr.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sr_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert set(api.EXPORTS) <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    seen = {sr.status_string(i) for i in range(7)}
+    assert len(seen) == 7 and sr.status_string(0) == "ok" and sr.status_string(99) == "unknown status"
+
+
+def _dims(**kw):
+    base = dict(n=1, c=3, h=4, w=4, scale=2, k=5, D=8)
+    base.update(kw)
+    return api.sr_dims(*(base[f] for f in ("n", "c", "h", "w", "scale", "k", "D")))
+
+
+FAKE = 0x1000  # never dereferenced: every call below fails validation before any launch
+
+
+def test_validation_errors_come_back_before_any_launch(lib):
+    dense = lambda d, coef=FAKE, dt=api.SR_F16, flags=0, lr=FAKE: lib.sr_dict_regress_dense(
+        lr, coef, dt, FAKE, FAKE, ctypes.byref(d), flags, None)
+    assert dense(_dims(), lr=None) == api.SR_ERR_NULL
+    assert dense(_dims(k=4)) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(k=11)) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(scale=0)) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(scale=9)) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(D=257)) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(D=0)) == api.SR_ERR_SHAPE
+    assert dense(_dims(n=0)) == api.SR_ERR_SHAPE
+    assert dense(_dims(h=70000, w=70000)) == api.SR_ERR_SHAPE
+    assert dense(_dims(), dt=7) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(), flags=api.SR_IDX_GLOBAL) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(), coef=FAKE + 1) == api.SR_ERR_ALIGN
+    assert dense(_dims(), coef=FAKE + 2, dt=api.SR_F32) == api.SR_ERR_ALIGN
+    assert lib.sr_dict_regress_dense(FAKE, FAKE, api.SR_F16, FAKE, FAKE, None, 0, None) == api.SR_ERR_NULL
+
+    assert lib.sr_bicubic_upsample(None, FAKE, ctypes.byref(_dims()), None) == api.SR_ERR_NULL
+    assert lib.sr_bicubic_upsample(FAKE, FAKE + 2, ctypes.byref(_dims()), None) == api.SR_ERR_ALIGN
+    assert lib.sr_bicubic_upsample(FAKE, FAKE, ctypes.byref(_dims(scale=12)), None) == api.SR_ERR_UNSUPPORTED
+
+    select = lambda d, s, flags=0, idx=FAKE: lib.sr_dict_select(FAKE, api.SR_F16, idx, None, ctypes.byref(d), s, flags, None)
+    assert select(_dims(), 0) == api.SR_ERR_SHAPE
+    assert select(_dims(), 9) == api.SR_ERR_SHAPE
+    assert select(_dims(), 4, flags=1) == api.SR_ERR_UNSUPPORTED
+    assert select(_dims(), 4, idx=None) == api.SR_ERR_NULL
+
+    selected = lambda d, s, flags=0, idx=FAKE, gamma=None: lib.sr_dict_regress_selected(
+        FAKE, FAKE, api.SR_F16, idx, gamma, FAKE, FAKE, ctypes.byref(d), s, flags, None)
+    assert selected(_dims(), 9) == api.SR_ERR_SHAPE
+    assert selected(_dims(), 4, flags=api.SR_IDX_GLOBAL, idx=None) == api.SR_ERR_NULL
+    assert selected(_dims(), 4, flags=api.SR_COEF_COMPACT, idx=None) == api.SR_ERR_NULL
+    assert selected(_dims(), 4, gamma=FAKE) == api.SR_ERR_UNSUPPORTED  # gamma only exists for the global subset
+    assert selected(_dims(), 4, flags=64) == api.SR_ERR_UNSUPPORTED
+    assert lib.sr_device_status(None, None) == api.SR_ERR_NULL
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    with pytest.raises(TypeError):
+        sr.sr_bicubic_upsample(torch.zeros(1, 1, 2, 2), 2)
