@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the dictionary-regression hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1]
+
+One step = one pass of the whole hot path over one frame batch of the workload (default: the
+1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. five library
+calls on one stream:
+    dense      sr_dict_regress_dense                         (up-sample + assemble + filter, fused)
+    select     sr_dict_select (indices + selected values)
+    compact    sr_dict_regress_selected from those index / value planes
+    fused      sr_dict_regress_selected with idx = NULL      (select + regress in one call)
+    global     sr_dict_regress_selected with one atom subset + re-weights (the paper's structured form)
+`value` is HR megapixels per second of whole steps (all N GPUs together; every rank owns its own
+frames and nothing is exchanged: weak scaling, no collective on the data path). Per-path times, the
+roofline of the dominant kernel and the CPU oracle timed on a bounded sample are reported beside it.
+
+`--impl reference` times the CPU oracle (test infrastructure, fp64, as it stands) on the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+PATHS = ("dense", "select", "compact", "fused", "global")
+METRIC = "HR megapixels/s"
+
+
+def algorithmic_bytes_per_pixel(wl, path: str) -> float:
+    """Bytes that must cross HBM per HR pixel: coefficients read once, output written once, LR read once."""
+    cb = 2 if wl.coef_dtype == "f16" else 4
+    io = 4 * wl.c + 4 * wl.c / (wl.scale ** 2)
+    s, D = wl.s, wl.D
+    return {
+        "dense": D * cb + io,
+        "select": D * cb + s + s * cb,            # read all planes, write uint8 indices and selected values
+        "compact": s * (cb + 1) + io,             # read index + value planes
+        "fused": D * cb + io,
+        "global": s * cb + io,                    # only the subset's planes are read
+    }[path]
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
+# kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": None, "select": None, "compact": None, "fused": None, "global": None}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid: str | None):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        if gpu_uuid:
+            cmd += ["-i", gpu_uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        # the busiest half of the samples: the sampler also sees the idle time around the timed region
+        busy = sorted(sm)[len(sm) // 2:] if sm else []
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_step(oracle, wl, lr, dict_, coef, S, gamma, rows: int | None, threads: int = 0):
+    """The step's five paths on the CPU oracle, on the top `rows` LR rows of every frame (None = all)."""
+    if rows is not None and rows < wl.h:
+        lr = lr[:, :, :rows].copy()
+        coef = coef[:, :, : rows * wl.scale].copy()
+    r, k, s = wl.scale, wl.k, wl.s
+    oracle.dict_regress_dense(lr, coef, dict_, r, k, flags=oracle.CLAMP01, threads=threads)
+    idx, sel = oracle.dict_select(coef, s, want_sel=True, threads=threads)
+    sel = sel.astype(coef.dtype)
+    oracle.dict_regress_selected(lr, sel, idx, None, dict_, r, k, s, flags=oracle.CLAMP01 | oracle.COEF_COMPACT, threads=threads)
+    oracle.dict_regress_selected(lr, coef, None, None, dict_, r, k, s, flags=oracle.CLAMP01, threads=threads)
+    oracle.dict_regress_selected(lr, coef, S, gamma, dict_, r, k, s, flags=oracle.CLAMP01 | oracle.IDX_GLOBAL, threads=threads)
+    return lr.shape[0] * lr.shape[2] * r * lr.shape[3] * r  # HR pixels processed
+
+
+def time_oracle(wl, lr, dict_, coef, S, gamma, budget_s: float = 20.0):
+    """Times the oracle on a bounded sample: a band of LR rows sized for roughly `budget_s` seconds."""
+    import oracle
+    probe_rows = max(1, min(wl.h, 8))
+    t0 = time.perf_counter()
+    px = oracle_step(oracle, wl, lr[:1], dict_, coef[:1], S, gamma, probe_rows)
+    dt = time.perf_counter() - t0
+    rate = px / dt
+    rows = int(max(probe_rows, min(wl.h, budget_s * rate / (wl.W * wl.scale))))
+    t0 = time.perf_counter()
+    px = oracle_step(oracle, wl, lr[:1], dict_, coef[:1], S, gamma, rows)
+    dt = time.perf_counter() - t0
+    return {"value": px / dt / 1e6, "unit": METRIC, "cores": oracle.max_threads(), "kind": "oracle",
+            "sample": f"top {rows} of {wl.h} LR rows of one frame ({px} HR pixels), all five paths of a step, "
+                      f"{dt:.2f} s of fp64 CPU work"}
+
+
+def run_reference(args, wl):
+    """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    import numpy as np
+    import sr_inputs
+    one = sr_inputs.Workload(wl.name, 1, wl.c, wl.h, wl.w, wl.scale, wl.D, wl.k, wl.coef_dtype, wl.s)
+    lr, dict_, coef = sr_inputs.make_inputs(one)
+    S = np.arange(0, wl.D, max(1, wl.D // wl.s), dtype=np.uint8)[: wl.s]
+    gamma = np.linspace(0.75, 1.25, wl.s).astype(np.float32)
+    # size a step so that warmup + steps end within a few minutes
+    t0 = time.perf_counter()
+    px = oracle_step(oracle, one, lr, dict_, coef, S, gamma, 4)
+    rate = px / (time.perf_counter() - t0)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rows = int(max(1, min(wl.h, budget * rate / (wl.W * wl.scale))))
+    for _ in range(args.warmup):
+        oracle_step(oracle, one, lr, dict_, coef, S, gamma, rows)
+    t0 = time.perf_counter()
+    px = 0
+    for _ in range(args.steps):
+        px += oracle_step(oracle, one, lr, dict_, coef, S, gamma, rows)
+    dt = time.perf_counter() - t0
+    value = px / dt / 1e6
+    sample = f"top {rows} of {wl.h} LR rows of one frame per step, all five paths"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "MP/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl),
+        "cpu_baseline": {"value": value, "unit": "MP/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "MP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(wl):
+    return {"workload": f"{wl.name}: LR {wl.n}x{wl.c}x{wl.h}x{wl.w} fp32, x{wl.scale} -> {wl.H}x{wl.W}, D={wl.D} atoms "
+                        f"of {wl.k}x{wl.k}, coefficients {wl.coef_dtype} [n][D][H][W], top-s s={wl.s}",
+            "paths_per_step": list(PATHS),
+            "l2": "coefficient tensor per frame is larger than the 126 MB L2 and three buffer sets rotate between steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    import sr_inputs
+    wl = sr_inputs.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import numpy as np
+    import torch
+    import paper_2303_08999_b200 as sr
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sr.load_library()
+
+    # ---- inputs: every rank owns its own frames (seed offset by rank); three rotating buffer sets
+    seed = sr_inputs.BASE_SEED + rank
+    lr, dict_, coef = sr_inputs.make_inputs(wl, seed)
+    S = np.arange(0, wl.D, max(1, wl.D // wl.s), dtype=np.uint8)[: wl.s]
+    gamma = np.linspace(0.75, 1.25, wl.s).astype(np.float32)
+    nsets = 3
+    h_lr = torch.from_numpy(lr).pin_memory()
+    h_coef = torch.from_numpy(coef).pin_memory()
+    d_dict, d_S, d_gamma = (torch.from_numpy(a).cuda() for a in (dict_, S, gamma))
+    sets = []
+    for _ in range(nsets):
+        sets.append({"lr": h_lr.cuda(non_blocking=True), "coef": h_coef.cuda(non_blocking=True)})
+    shape_out = (wl.n, wl.c, wl.H, wl.W)
+    outs = {p: torch.empty(shape_out, dtype=torch.float32, device="cuda") for p in ("dense", "compact", "fused", "global")}
+    idx = torch.empty((wl.n, wl.s, wl.H, wl.W), dtype=torch.uint8, device="cuda")
+    sel = torch.empty((wl.n, wl.s, wl.H, wl.W), dtype=h_coef.dtype, device="cuda")
+    flags = sr.SR_CLAMP01
+    r, k, s = wl.scale, wl.k, wl.s
+    torch.cuda.synchronize()
+
+    def step(bufs, events=None):
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                events.append(e)
+        mark()
+        sr.sr_dict_regress_dense(bufs["lr"], bufs["coef"], d_dict, r, k, flags, out=outs["dense"])
+        mark()
+        sr.sr_dict_select(bufs["coef"], s, idx=idx, sel=sel)
+        mark()
+        sr.sr_dict_regress_selected(bufs["lr"], sel, idx, None, d_dict, r, k, s, flags | sr.SR_COEF_COMPACT, out=outs["compact"])
+        mark()
+        sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], None, None, d_dict, r, k, s, flags, out=outs["fused"])
+        mark()
+        sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], d_S, d_gamma, d_dict, r, k, s, flags | sr.SR_IDX_GLOBAL, out=outs["global"])
+        mark()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(sets[i % nsets])
+    barrier()
+
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    launches0 = sr.sr_launch_count()
+    events = []
+    barrier()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(args.steps):
+        step(sets[i % nsets], events)
+    t_end.record()
+    barrier()
+    elapsed_ms = t_start.elapsed_time(t_end)
+    launches = sr.sr_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    if sr.sr_device_status() != 0:
+        raise SystemExit("device status word reports an expired wait")
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+
+    # per-path averages from the events recorded inside the timed region
+    per_path_ms = {}
+    per = len(PATHS) + 1
+    for j, p in enumerate(PATHS):
+        ts = [events[i * per + j].elapsed_time(events[i * per + j + 1]) for i in range(args.steps)]
+        per_path_ms[p] = sum(ts) / len(ts)
+
+    # ---- end to end through the public API with host buffers: pinned H2D of the step's inputs, D2H of its results
+    e2e = None
+    if not args.no_e2e:
+        h_out = {p: torch.empty(shape_out, dtype=torch.float32).pin_memory() for p in outs}
+        bufs = sets[0]
+        e2e_steps = max(3, min(args.steps, 10))
+
+        def e2e_step():
+            bufs["lr"].copy_(h_lr, non_blocking=True)
+            bufs["coef"].copy_(h_coef, non_blocking=True)
+            step(bufs)
+            for p in outs:
+                h_out[p].copy_(outs[p], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * wl.npix * e2e_steps / (ms * 1e-3) / 1e6, "unit": "MP/s",
+               "h2d_bytes_per_step": h_lr.numel() * 4 + h_coef.numel() * h_coef.element_size(),
+               "d2h_bytes_per_step": sum(o.numel() * 4 for o in outs.values()), "steps": e2e_steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = load_peaks()
+    paths = {}
+    for p in PATHS:
+        by = algorithmic_bytes_per_pixel(wl, p) * wl.npix
+        gbs = by / (per_path_ms[p] * 1e-3) / 1e9
+        paths[p] = {"ms": per_path_ms[p], "mp_per_s": wl.npix / (per_path_ms[p] * 1e-3) / 1e6,
+                    "frames_per_s": wl.n / (per_path_ms[p] * 1e-3), "algorithmic_bytes": by, "achieved_gbs": gbs,
+                    "frac_of_hbm": gbs / peak}
+    dominant = max(PATHS, key=lambda p: per_path_ms[p])
+    tr = NCU_TRAFFIC_BYTES_PER_PIXEL.get(dominant)
+    roofline = {"kernel": dominant, "bound": "hbm", "achieved": paths[dominant]["achieved_gbs"], "peak": peak,
+                "unit": "GB/s", "frac": paths[dominant]["frac_of_hbm"], "peak_kind": f"of {peak_kind}",
+                "traffic": None if tr is None else tr * wl.npix}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = time_oracle(wl, lr, dict_, coef, S, gamma)
+
+    line = {
+        "metric": METRIC, "value": world * wl.npix * args.steps / (elapsed_ms * 1e-3) / 1e6, "unit": "MP/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate, f16 coefficients"
+        if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": workload_config(wl),
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
+        "paths": paths,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

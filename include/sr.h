@@ -126,6 +126,12 @@ const char* sr_status_string(int status);
  */
 int sr_device_status(void* stream, int* out_status);
 
+/*
+ * Number of kernels this library has launched in this process so far (all devices, all streams).
+ * Introspection for benchmarks and tests; the paper has no counterpart.
+ */
+int64_t sr_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

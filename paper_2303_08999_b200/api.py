@@ -20,7 +20,7 @@ SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT = 1, 2, 4
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
-           "sr_status_string", "sr_device_status")
+           "sr_status_string", "sr_device_status", "sr_launch_count")
 
 
 class sr_dims(ctypes.Structure):
@@ -52,6 +52,8 @@ def load_library() -> ctypes.CDLL:
         lib.sr_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
         for name in EXPORTS:
             getattr(lib, name).restype = i32
+        lib.sr_launch_count.argtypes = []
+        lib.sr_launch_count.restype = ctypes.c_int64
         lib.sr_status_string.argtypes = [i32]
         lib.sr_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -163,3 +165,8 @@ def sr_device_status() -> int:
     v = ctypes.c_int(0)
     _check(load_library().sr_device_status(_stream(), ctypes.byref(v)), "sr_device_status")
     return v.value
+
+
+def sr_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().sr_launch_count())

@@ -1,12 +1,17 @@
 // C ABI entry points: argument validation, path selection, status reporting.
 #include <math.h>
 
+#include <atomic>
+
 #include "sr_common.cuh"
 #include "sr_umma.cuh"
 
 namespace sr {
 
 __device__ int g_status_word = 0;
+
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 int* device_status_word()
 {
@@ -164,6 +169,8 @@ const char* sr_status_string(int status)
     default: return "unknown status";
     }
 }
+
+int64_t sr_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 int sr_device_status(void* stream, int* out_status)
 {

@@ -40,6 +40,7 @@ cudaError_t launch_bicubic(const float* lr, float* hr, const Problem& pb, cudaSt
     const int64_t cap = 148 * 8 * 4;
     if (blocks > cap) blocks = cap;
     bicubic_kernel<<<(unsigned)blocks, 256, 0, st>>>(lr, hr, pb);
+    count_launches(1);
     return cudaGetLastError();
 }
 

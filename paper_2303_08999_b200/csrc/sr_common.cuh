@@ -41,6 +41,9 @@ BicubicPhases make_phases(int scale);
 // Address of the per-device status word (device memory; 0 = ok). Returns nullptr on a CUDA error.
 int* device_status_word();
 
+// Adds to the process-wide count of kernels launched (read back by sr_launch_count).
+void count_launches(int n);
+
 // Launchers. Each returns a cudaError_t from the launch.
 cudaError_t launch_bicubic(const float* lr, float* hr, const Problem& pb, cudaStream_t st);
 cudaError_t launch_regress_fma(int mode, const float* lr, const void* coef, int coef_dtype, const uint8_t* idx,

@@ -135,6 +135,7 @@ cudaError_t launch_t(const float* lr, const void* coef, const uint8_t* idx, cons
     dim3 grid((pb.W + TX - 1) / TX, (pb.H + TY - 1) / TY, pb.n), block(TX, TY);
     if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidConfiguration;
     kern<<<grid, block, smem, st>>>(lr, (const CoefT*)coef, idx, gamma, dict, out, pb);
+    count_launches(1);
     return cudaGetLastError();
 }
 

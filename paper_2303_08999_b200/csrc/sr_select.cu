@@ -94,6 +94,7 @@ cudaError_t launch_sel(const void* coef, uint8_t* idx, void* sel, const Problem&
     else if (pb.s <= 8) select_insert_kernel<CoefT, 8><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
     else if (pb.s <= 16) select_insert_kernel<CoefT, 16><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
     else select_scan_kernel<CoefT><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
+    count_launches(1);
     return cudaGetLastError();
 }
 
