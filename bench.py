@@ -196,10 +196,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--paths", default=",".join(PATHS), help="comma-separated subset of the step's paths (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    active = tuple(p for p in PATHS if p in args.paths.split(","))
+    if "compact" in active and "select" not in active:
+        active = tuple(p for p in PATHS if p in active or p == "select")   # compact consumes select's outputs
 
     import sr_inputs
     wl = sr_inputs.CONFIGS[args.workload]
@@ -250,15 +254,20 @@ def main():
                 e.record()
                 events.append(e)
         mark()
-        sr.sr_dict_regress_dense(bufs["lr"], bufs["coef"], d_dict, r, k, flags, out=outs["dense"])
+        if "dense" in active:
+            sr.sr_dict_regress_dense(bufs["lr"], bufs["coef"], d_dict, r, k, flags, out=outs["dense"])
         mark()
-        sr.sr_dict_select(bufs["coef"], s, idx=idx, sel=sel)
+        if "select" in active:
+            sr.sr_dict_select(bufs["coef"], s, idx=idx, sel=sel)
         mark()
-        sr.sr_dict_regress_selected(bufs["lr"], sel, idx, None, d_dict, r, k, s, flags | sr.SR_COEF_COMPACT, out=outs["compact"])
+        if "compact" in active:
+            sr.sr_dict_regress_selected(bufs["lr"], sel, idx, None, d_dict, r, k, s, flags | sr.SR_COEF_COMPACT, out=outs["compact"])
         mark()
-        sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], None, None, d_dict, r, k, s, flags, out=outs["fused"])
+        if "fused" in active:
+            sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], None, None, d_dict, r, k, s, flags, out=outs["fused"])
         mark()
-        sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], d_S, d_gamma, d_dict, r, k, s, flags | sr.SR_IDX_GLOBAL, out=outs["global"])
+        if "global" in active:
+            sr.sr_dict_regress_selected(bufs["lr"], bufs["coef"], d_S, d_gamma, d_dict, r, k, s, flags | sr.SR_IDX_GLOBAL, out=outs["global"])
         mark()
 
     def barrier():
@@ -340,13 +349,13 @@ def main():
 
     peak, peak_kind = load_peaks()
     paths = {}
-    for p in PATHS:
+    for p in active:
         by = algorithmic_bytes_per_pixel(wl, p) * wl.npix
         gbs = by / (per_path_ms[p] * 1e-3) / 1e9
         paths[p] = {"ms": per_path_ms[p], "mp_per_s": wl.npix / (per_path_ms[p] * 1e-3) / 1e6,
                     "frames_per_s": wl.n / (per_path_ms[p] * 1e-3), "algorithmic_bytes": by, "achieved_gbs": gbs,
                     "frac_of_hbm": gbs / peak}
-    dominant = max(PATHS, key=lambda p: per_path_ms[p])
+    dominant = max(active, key=lambda p: per_path_ms[p])
     tr = NCU_TRAFFIC_BYTES_PER_PIXEL.get(dominant)
     roofline = {"kernel": dominant, "bound": "hbm", "achieved": paths[dominant]["achieved_gbs"], "peak": peak,
                 "unit": "GB/s", "frac": paths[dominant]["frac_of_hbm"], "peak_kind": f"of {peak_kind}",
@@ -360,7 +369,7 @@ def main():
         "metric": METRIC, "value": world * wl.npix * args.steps / (elapsed_ms * 1e-3) / 1e6, "unit": "MP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate, f16 coefficients"
-        if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": workload_config(wl),
+        if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": dict(workload_config(wl), paths_per_step=list(active)),
         "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
         "paths": paths,
     }
