@@ -36,19 +36,24 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
                  : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+// One try: the hardware may park the thread for up to ~`hint_ns` before answering, which keeps a waiting
+// warp out of the issue slots without delaying its wake-up when the phase completes.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns = 2000u)
 {
     uint32_t done;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
         : "memory");
     return done != 0;
 }
 
 // Cycle budget of one wait (about a second at B200 clocks).
 constexpr long long kWaitCycleLimit = 1ll << 31;
+
+// Whole-warp wait: lane 0 polls, the result is broadcast. Returns the same value in every lane.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag);
 
 // Waits for the phase with the given parity to complete. Returns false when the budget ran out or
 // another thread of the CTA has already raised `*abort_flag` (a shared-memory word).
@@ -64,6 +69,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             return false;
         }
     }
+}
+
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    // lanes other than 0 did not observe the barrier themselves: one successful test gives them the acquire
+    if (ok) while (!mbar_try_wait(bar, parity, 0u)) {}
+    return ok != 0;
 }
 
 // ---- proxies / fences ----------------------------------------------------------------------------------------------
@@ -158,6 +173,49 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, float* v)
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_x8(uint32_t taddr, float* v)
+{
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_x4(uint32_t taddr, float* v)
+{
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_x1(uint32_t taddr, float* v)
+{
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r[0]) : "r"(taddr) : "memory");
+}
+
+// Loads N (1..16) consecutive columns with the fewest instructions of width 16, 8, 4, 1.
+template <int N>
+__device__ __forceinline__ void tmem_ld_n(uint32_t taddr, float* v)
+{
+    if constexpr (N >= 16) {
+        tmem_ld_x16(taddr, v);
+        if constexpr (N > 16) tmem_ld_n<N - 16>(taddr + 16, v + 16);
+    } else if constexpr (N >= 8) {
+        tmem_ld_x8(taddr, v);
+        if constexpr (N > 8) tmem_ld_n<N - 8>(taddr + 8, v + 8);
+    } else if constexpr (N >= 4) {
+        tmem_ld_x4(taddr, v);
+        if constexpr (N > 4) tmem_ld_n<N - 4>(taddr + 4, v + 4);
+    } else if constexpr (N >= 1) {
+        tmem_ld_x1(taddr, v);
+        if constexpr (N > 1) tmem_ld_n<N - 1>(taddr + 1, v + 1);
+    }
 }
 
 } // namespace ptx

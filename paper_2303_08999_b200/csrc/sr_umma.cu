@@ -1,23 +1,27 @@
-// Fused regression kernel for sm_100a: TMA-streamed coefficient planes, dictionary assembly F = Phi D on the
-// tcgen05 tensor cores with fp32 accumulators in tensor memory, bicubic tile + patch dot product + clamp in the
-// epilogue. The filter matrix F (TMEM / registers), the up-sampled image U and its patches (shared memory) never
-// reach HBM: per HR pixel the kernel reads its coefficients once and writes its c output values once.
+// Fused regression kernel for sm_100a: coefficient planes streamed with 16-byte asynchronous copies, dictionary
+// assembly F = Phi D on the tcgen05 tensor cores with fp32 accumulators in tensor memory, bicubic tile + patch dot
+// product + clamp in the epilogue. The filter matrix F (TMEM / registers), the up-sampled image U and its patches
+// (shared memory) never reach HBM: per HR pixel the kernel reads its coefficients once and writes its c output
+// values once.
 //
-// One persistent CTA per SM walks HR tiles of 128 x 8 pixels. A tile row (128 pixels of one HR row) is one
-// pipeline stage: two TMA boxes of [atoms][64 pixels] binary16 land in shared memory in the 128-byte-swizzled
-// MN-major layout the tensor core reads directly (pixels are M, atoms are K), so the planar [n][D][H][W]
-// coefficient tensor needs no transpose. The dictionary is the B operand (K-major): its fp32 values are split
-// into binary16 hi + lo parts (~22 bits kept) that sit side by side along N, so one MMA per 16 atoms reads the
-// coefficient stage once and yields both partial filters; the epilogue adds them. N = 2 x (k*k padded to 16).
+// One persistent CTA per SM walks HR tiles of 128 x 16 pixels. A tile row (128 pixels of one HR row) is one
+// pipeline stage [atoms][128 pixels] binary16, written by cp.async.cg (coalesced 128-bit loads, L1 bypassed)
+// straight into the 128-byte-swizzled MN-major layout the tensor core reads (pixels are M, atoms are K), so the
+// planar [n][D][H][W] coefficient tensor needs no transpose. (A TMA box over 72 planes 4 MB apart streams at
+// ~4.2 TB/s on B200; the same bytes through cp.async reach ~5.5 TB/s, hence this choice.) The dictionary is the
+// B operand (K-major): its fp32 values are split into binary16 hi + lo parts (~22 bits kept) that sit side by
+// side along N, so one MMA per 16 atoms reads the coefficient stage once and yields both partial filters; the
+// epilogue adds them. N = 2 x (k*k padded to 16).
 //
-// Shared-memory bandwidth is the scarce on-chip resource here (TMA fill + operand reads + U tile + patch reads),
-// so the epilogue keeps a sliding k x k x 3 window of U in registers and reads each U row once per pixel column.
+// Shared-memory bandwidth and per-warp latency are the scarce on-chip resources, so the epilogue keeps a sliding
+// k x k x 3 window of U in registers and reads each U row once per pixel column.
 //
-// Warp roles (448 threads):
-//   warp 0       TMA producer            full[stage]  <- bytes landed        waits empty[stage]
-//   warp 1       MMA issuer, TMEM owner  acc_full[a], empty[stage] <- tcgen05.commit; waits full[stage], acc_empty[a]
-//   warps 2-9    U producers             bicubic (separable) of the tile + halo into a double-buffered tile
-//   warps 10-13  epilogue                TMEM -> registers (one pixel's filter per thread), patch dot, clamp, store
+// Warp roles (512 threads):
+//   warps 0-3    coefficient producers   full[stage] <- cp.async arrivals when the copies land; wait empty[stage]
+//   warp 4       MMA issuer, TMEM owner  acc_full[a], empty[stage] <- tcgen05.commit; waits full[stage], acc_empty[a]
+//   warps 5-7    U producers             bicubic (separable) of the tile + halo into a double-buffered tile
+//   warps 8-15   epilogue (2 x 4 warps)  TMEM -> registers (one pixel's filter per thread), patch dot, clamp, store;
+//                                        the two groups own the upper and the lower half of a tile
 // Every wait is bounded; on expiry the CTA raises its abort flag, sets the device status word and drains.
 #include "sr_ptx.cuh"
 #include "sr_umma.cuh"
@@ -28,9 +32,10 @@ namespace {
 
 using namespace ptx;
 
-constexpr int TW = 128, TH = 8;
-constexpr int kThreads = 448;
-constexpr int kFirstUWarp = 2, kNumUWarps = 8, kFirstEpiWarp = 10, kNumEpiWarps = 4;
+constexpr int TW = 128, TH = 16;
+constexpr int kThreads = 512;
+constexpr int kNumLoadWarps = 4, kMmaWarp = 4;
+constexpr int kFirstUWarp = 5, kNumUWarps = 3, kFirstEpiWarp = 8, kNumEpiWarps = 8;
 constexpr int kMaxStages = 8;
 constexpr int kMaxAccSlots = 8;
 constexpr int kMaxChannels = 4;
@@ -47,7 +52,9 @@ struct UmmaParams {
     int mode;
     int natoms;           // coefficient planes per pixel that enter the contraction (D, or s for a subset)
     int dpad;             // natoms rounded up to a multiple of 16 (the MMA K extent)
-    int per_atom_boxes;   // 1: one TMA box per selected atom (subset of a full tensor); 0: one box covers all atoms
+    int planes;           // planes per frame in the coefficient tensor (D, or s when it is compact)
+    int gather_planes;    // 1: plane q of the contraction is plane atoms[q] of the tensor (subset of a full tensor)
+    const __half* coef;
     int stages;
     int trows;            // LR rows a tile can need (rows of the horizontal-pass scratch tile)
     int tcols;            // LR columns a tile can need
@@ -65,7 +72,7 @@ struct __align__(16) Ctl {
     float4 vy_w[TH + 2 * 4];   // per U-tile row: its four vertical tap weights
     float4 hx_w[TW + 2 * 4];   // per U-tile column: its four horizontal tap weights
     int vy_off[TH + 2 * 4];    // per U-tile row: first row of the scratch tile it reads
-    int hx_off[TW + 2 * 4];    // per U-tile column: first column of the LR window it reads
+    alignas(16) int hx_off[TW + 2 * 4];   // per U-tile column: first column of the LR window it reads
     uint8_t atoms[256];        // subset mode: the atom id of each selected plane
 };
 
@@ -74,7 +81,8 @@ template <int K> struct Geo {
     static constexpr int NPAD = (kk + 15) / 16 * 16;     // taps padded; hi part in columns [0, NPAD), lo in [NPAD, 2 NPAD)
     static constexpr int NB = 2 * NPAD;                  // N of the MMA
     static constexpr int P = (K - 1) / 2;
-    static constexpr int UW = TW + 2 * P, UH = TH + 2 * P;
+    static constexpr int UW = (TW + 2 * P + 3) & ~3;     // U tile width: tile + halo, rounded up to 4 for 16-byte rows
+    static constexpr int UH = TH + 2 * P;
     static constexpr int LBO_B = (NB / 8) * 128;         // bytes between the two K-halves of a K-step of the B operand
     static constexpr int KSTEP_B = 2 * LBO_B;            // bytes per K-step (16 atoms) of the B operand
     static constexpr int ACC_SLOTS = (512 / NB) < kMaxAccSlots ? (512 / NB) : kMaxAccSlots;
@@ -94,6 +102,17 @@ __device__ __forceinline__ void decode_tile(const UmmaParams& p, int t, int& f, 
     rows = min(TH, p.pb.H - y0);
 }
 
+// Rows of a tile are streamed in the order 0, H, 1, H+1, ... (H = TH/2) so that the two epilogue groups, which
+// own the upper and the lower half of the tile, both receive work from the start. Item i of a tile with `rows`
+// valid rows maps to a tile row; every role enumerates the same sequence.
+constexpr int kHalf = TH / 2;
+__device__ __forceinline__ int tile_row_of_item(int i, int rows)
+{
+    const int h1 = rows > kHalf ? rows - kHalf : 0;      // rows in the lower half
+    // the first 2*h1 items alternate between the halves, the rest belong to the upper half
+    return i < 2 * h1 ? ((i & 1) ? kHalf + (i >> 1) : (i >> 1)) : i - h1;
+}
+
 // LR pixels a tile (plus patch halo) needs for its bicubic taps: rows lr_lo .. lr_lo + nrows - 1 and columns
 // col_lo .. col_lo + ncols - 1 (unclamped; reads clamp them to the image).
 struct LrWindow { int f, y0, x0, rows, lr_lo, nrows, col_lo, ncols; };
@@ -108,7 +127,7 @@ __device__ __forceinline__ void lr_window(const UmmaParams& p, int t, LrWindow& 
     const int qylo = fast_div(Ylo, pb.r, p.r_magic), qyhi = fast_div(Yhi, pb.r, p.r_magic);
     g.lr_lo = qylo + pb.ph.base[Ylo - qylo * pb.r];
     g.nrows = qyhi + pb.ph.base[Yhi - qyhi * pb.r] + 3 - g.lr_lo + 1;      // <= trows
-    const int Xlo = clampi(g.x0 - P, 0, pb.W - 1), Xhi = clampi(g.x0 + TW - 1 + P, 0, pb.W - 1);
+    const int Xlo = clampi(g.x0 - P, 0, pb.W - 1), Xhi = clampi(g.x0 - P + Geo<K>::UW - 1, 0, pb.W - 1);
     const int qxlo = fast_div(Xlo, pb.r, p.r_magic), qxhi = fast_div(Xhi, pb.r, p.r_magic);
     g.col_lo = qxlo + pb.ph.base[Xlo - qxlo * pb.r];
     g.ncols = qxhi + pb.ph.base[Xhi - qxhi * pb.r] + 3 - g.col_lo + 1;     // <= tcols
@@ -118,8 +137,34 @@ __device__ __forceinline__ void cp_async_f32(float* dst_smem, const float* src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
 }
+// 16-byte copy global -> shared, L1 bypassed; src_bytes = 0 writes zeros instead of reading.
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+// Arrives on the mbarrier (without raising its pending count) once all cp.async of this thread so far completed.
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint64_t* bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// cp.async.wait_group with a run-time count (0..7): at most n of this thread's groups remain in flight.
+__device__ __forceinline__ void cp_async_wait_dyn(int n)
+{
+    switch (n) {
+    case 0: cp_async_wait<0>(); break;
+    case 1: cp_async_wait<1>(); break;
+    case 2: cp_async_wait<2>(); break;
+    case 3: cp_async_wait<3>(); break;
+    case 4: cp_async_wait<4>(); break;
+    case 5: cp_async_wait<5>(); break;
+    case 6: cp_async_wait<6>(); break;
+    default: cp_async_wait<7>(); break;
+    }
+}
 
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads)
 {
@@ -138,21 +183,26 @@ __device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pre
     return r != 0;
 }
 
-// One pixel's filter from tensor memory: F[j] = hi[j] + lo[j] for the taps j < k*k (16 columns at a time).
+// One pixel's filter from tensor memory: F[j] = hi[j] + lo[j] for the taps j < k*k (at most 16 columns at a time).
 template <int K>
 __device__ __forceinline__ void load_filter(uint32_t taddr, float* F)
 {
     using G = Geo<K>;
 #pragma unroll
-    for (int j0 = 0; j0 < G::NPAD; j0 += 16) {
-        if (j0 < G::kk) {
-            float h[16], l[16];
-            tmem_ld_x16(taddr + j0, h);
-            tmem_ld_x16(taddr + G::NPAD + j0, l);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) F[j0 + i] = h[i] + l[i];
+    for (int j0 = 0; j0 < G::kk; j0 += 16) {
+        constexpr int kTail = G::kk % 16;
+        float h[16], l[16];
+        if (j0 + 16 <= G::kk) {
+            tmem_ld_n<16>(taddr + j0, h);
+            tmem_ld_n<16>(taddr + G::NPAD + j0, l);
+        } else {
+            tmem_ld_n<kTail ? kTail : 16>(taddr + j0, h);
+            tmem_ld_n<kTail ? kTail : 16>(taddr + G::NPAD + j0, l);
         }
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (j0 + i < G::kk) F[j0 + i] = h[i] + l[i];
     }
 }
 
@@ -179,11 +229,83 @@ __device__ __forceinline__ void patch_dot(const float* F, const float* u, int ch
     }
 }
 
+struct EpiCtx {
+    int quarter, group, x;
+    int64_t HW;
+    bool clamp01;
+    uint32_t tmem_lane_base;
+};
+
+// Position in a tile's streaming order of row j of half `group` (inverse of tile_row_of_item).
+__device__ __forceinline__ int item_of_half_row(int j, int group, int h1)
+{
+    return j < h1 ? 2 * j + group : j + h1;              // beyond h1 only the upper half (group 0) has rows
+}
+
+// Epilogue of one half tile (rows j = 0 .. my_rows-1 of the half, top to bottom) for a three-channel image:
+// the k x k x 3 patch lives in registers as a sliding window (slot of U row u is u % K, all indices
+// compile-time), so each row costs 3 * K shared loads instead of 3 * K * K. Returns false when a wait expired.
+template <int K, class CtlT>
+__device__ __forceinline__ bool epilogue_half_windowed(CtlT& ctl, const EpiCtx& e, const float* Ub, float* dst0, int W,
+                                                       int my_rows, int h1, uint32_t it_base, bool in_x,
+                                                       volatile int* abort_flag)
+{
+    using G = Geo<K>;
+    float win[3][K][K];
+    const float* u0 = Ub + e.x;
+    bool ok = true;
+    if (my_rows > 0) {
+#pragma unroll
+        for (int u = 0; u < K - 1; ++u)
+#pragma unroll
+            for (int c = 0; c < 3; ++c)
+#pragma unroll
+                for (int b = 0; b < K; ++b) win[c][u][b] = u0[(c * G::UH + u) * G::UW + b];
+    }
+#pragma unroll
+    for (int j = 0; j < kHalf; ++j) {
+        if (j < my_rows && ok) {
+#pragma unroll
+            for (int c = 0; c < 3; ++c)
+#pragma unroll
+                for (int b = 0; b < K; ++b) win[c][(j + K - 1) % K][b] = u0[(c * G::UH + j + K - 1) * G::UW + b];
+            const uint32_t it = it_base + item_of_half_row(j, e.group, h1);
+            const int a_slot = it % G::ACC_SLOTS;
+            const uint32_t aph = (it / G::ACC_SLOTS) & 1;
+            ok = mbar_wait_warp(&ctl.acc_full[a_slot], aph, abort_flag);
+            if (ok) {
+                tc_fence_after_sync();
+                float F[G::NPAD];
+                load_filter<K>(e.tmem_lane_base + (uint32_t)(a_slot * G::NB), F);
+                tc_fence_before_sync();
+                mbar_arrive(&ctl.acc_empty[a_slot]);
+                float acc[3][2];
+#pragma unroll
+                for (int c = 0; c < 3; ++c) acc[c][0] = acc[c][1] = 0.f;
+#pragma unroll
+                for (int a = 0; a < K; ++a)
+#pragma unroll
+                    for (int b = 0; b < K; ++b)
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) acc[c][a & 1] = fmaf(F[a * K + b], win[c][(j + a) % K][b], acc[c][a & 1]);
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    float v = acc[c][0] + acc[c][1];
+                    if (e.clamp01) v = fminf(fmaxf(v, 0.f), 1.f);
+                    if (in_x) dst0[c * e.HW + (int64_t)j * W] = v;
+                }
+            }
+        }
+    }
+    return ok;
+}
+
 // Optional role timing (build with -DSR_PROFILE_ROLES): cycles each role spends in total and inside waits,
 // written per CTA to the buffer registered with sr_debug_role_profile.
 #ifdef SR_PROFILE_ROLES
 __device__ long long* g_role_prof = nullptr;
-#define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0, prof_tw = 0, prof_mma = 0, prof_commit = 0; bool prof_tmp_ok = true;
+__device__ int g_debug_mode = 0;   // 1: TMA streaming only (no MMA, no U, no epilogue)
+#define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0, prof_tw = 0, prof_mma = 0, prof_commit = 0, prof_a = 0, prof_b = 0, prof_c = 0, prof_d = 0; bool prof_tmp_ok = true;
 #define PROF_WAIT(expr) (prof_tw = clock64(), prof_tmp_ok = (expr), prof_wait += clock64() - prof_tw, prof_tmp_ok)
 #define PROF_T(var) long long var = clock64();
 #define PROF_ADD(acc, t0) acc += clock64() - (t0);
@@ -200,14 +322,16 @@ __device__ long long* g_role_prof = nullptr;
 
 template <int K>
 __global__ void __launch_bounds__(kThreads, 1)
-regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_constant__ CUtensorMap map_row,
-                    const __grid_constant__ UmmaParams p)
+regress_umma_kernel(const __grid_constant__ UmmaParams p)
 {
     using G = Geo<K>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ Ctl ctl;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef SR_PROFILE_ROLES
+    unsigned long long gt_entry; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_entry));
+#endif
     const Problem& pb = p.pb;
     const int C = pb.c;
     const int stage_bytes = p.dpad * 256;            // two chunks of [dpad][64 pixels] binary16
@@ -223,13 +347,11 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_co
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
-        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], 1); mbar_init(&ctl.empty[i], 1); }
-        for (int i = 0; i < kMaxAccSlots; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], kNumEpiWarps * 32); }
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], kNumLoadWarps * 32); mbar_init(&ctl.empty[i], 1); }
+        for (int i = 0; i < kMaxAccSlots; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], 128); }
         for (int i = 0; i < 2; ++i) { mbar_init(&ctl.u_full[i], kNumUWarps * 32); mbar_init(&ctl.u_empty[i], kNumEpiWarps * 32); }
         ctl.abort_flag = 0;
         fence_barrier_init();
-        prefetch_tensormap(&map_all);
-        prefetch_tensormap(&map_row);
     }
     // B operand: dict (or gamma-weighted subset rows) as binary16 hi | lo along N, K-major, no swizzle.
     // element (column n, atom k) of a K-step: (k%16)/8 * LBO + n/8 * 128 + n%8 * 16 + k%8 * 2
@@ -251,66 +373,78 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_co
         *reinterpret_cast<__half*>(sB + base + (n >> 3) * 128 + (n & 7) * 16) = hi;
         *reinterpret_cast<__half*>(sB + base + (nl >> 3) * 128 + (nl & 7) * 16) = lo;
     }
-    if (p.per_atom_boxes)
+    if (p.gather_planes)
         for (int q = tid; q < p.natoms; q += kThreads) ctl.atoms[q] = (uint8_t)min((int)__ldg(p.idx + q), pb.D - 1);
-    // Rows of the A stages that no TMA box writes (subset mode: atoms natoms..dpad-1) must read as zero.
-    if (p.per_atom_boxes) {
+    // The copies only ever write rows < natoms of a stage; the padding rows up to dpad must read as zero.
+    {
         uint4* a4 = reinterpret_cast<uint4*>(sA);
         const int n16 = p.stages * stage_bytes / 16;
         for (int i = tid; i < n16; i += kThreads) a4[i] = make_uint4(0, 0, 0, 0);
     }
     fence_proxy_async_smem();
     __syncwarp();
-    if (warp == 1) tmem_alloc(&ctl.tmem_base, G::TMEM_COLS);
+    if (warp == kMmaWarp) tmem_alloc(&ctl.tmem_base, G::TMEM_COLS);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl.tmem_base;
     volatile int* abort_flag = &ctl.abort_flag;
     PROF_DECL
+#ifdef SR_PROFILE_ROLES
+    unsigned long long gt_setup; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_setup));
+#endif
 
     // ---------------------------------------------------------------- roles
-    if (warp == 0) {
-        // ===== TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            int s = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
-                int f, y0, x0, rows;
-                decode_tile(p, t, f, y0, x0, rows);
-                for (int r = 0; r < rows; ++r, ++it) {
-                    if (!(ok = PROF_WAIT(mbar_wait(&ctl.empty[s], ph ^ 1, abort_flag)))) break;
-                    uint8_t* dst = sA + (size_t)s * stage_bytes;
-                    if (!p.per_atom_boxes) {
-                        mbar_arrive_expect_tx(&ctl.full[s], stage_bytes);
-                        tma_load_4d(dst, &map_all, &ctl.full[s], x0, y0 + r, 0, f);
-                        tma_load_4d(dst + chunk_bytes, &map_all, &ctl.full[s], x0 + 64, y0 + r, 0, f);
-                    } else {
-                        mbar_arrive_expect_tx(&ctl.full[s], p.natoms * 256);
-                        for (int q = 0; q < p.natoms; ++q) {
-                            const int a = ctl.atoms[q];
-                            tma_load_4d(dst + q * 128, &map_row, &ctl.full[s], x0, y0 + r, a, f);
-                            tma_load_4d(dst + chunk_bytes + q * 128, &map_row, &ctl.full[s], x0 + 64, y0 + r, a, f);
-                        }
+#ifdef SR_PROFILE_ROLES
+    const int debug_mode = g_debug_mode;
+    if (debug_mode >= 1 && warp > kMmaWarp) goto teardown;
+#endif
+    if (warp < kNumLoadWarps) {
+        // ===== coefficient producers: 128 threads, thread = (16-byte column c16 of the 128-pixel row, atom l0 + 8k)
+        // A stage is [chunk of 64 pixels][atom][128 B]; within a 1024-byte group of 8 atoms the 16-byte columns are
+        // XOR-swizzled with the atom index (the 128-byte swizzle the MMA descriptor names).
+        constexpr int NL = kNumLoadWarps * 32;
+        const int c16 = tid & 15, l0 = tid >> 4;             // l0 in 0..7: constant (l & 7) for this thread
+        const uint32_t dst_thread = (uint32_t)((c16 >> 3) * chunk_bytes + l0 * 128 + (((c16 & 7) ^ l0) << 4));
+        const int64_t plane_elems = (int64_t)pb.H * pb.W;
+        int s = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+            int f, y0, x0, rows;
+            decode_tile(p, t, f, y0, x0, rows);
+#ifdef SR_PROFILE_ROLES
+            if (debug_mode == 2) { int rr; decode_tile(p, blockIdx.x % p.tiles_x, f, y0, x0, rr); }   // L2-resident re-reads
+#endif
+            const int xe = x0 + c16 * 8;                     // first of this thread's 8 pixels
+            const uint32_t src_bytes = xe < pb.W ? 16u : 0u; // columns beyond the image are zero-filled
+            const __half* src_col = p.coef + (int64_t)f * p.planes * plane_elems + (xe < pb.W ? xe : 0);
+            for (int r = 0; r < rows; ++r) {
+                ok = PROF_WAIT(mbar_wait_warp(&ctl.empty[s], ph ^ 1, abort_flag));
+                if (!ok) break;
+                const int yr = y0 + tile_row_of_item(r, rows);
+                const __half* src_row = src_col + (int64_t)yr * pb.W;
+                uint32_t dst = smem_u32(sA + (size_t)s * stage_bytes) + dst_thread;
+                if (!p.gather_planes) {
+                    const __half* src = src_row + l0 * plane_elems;
+#pragma unroll 3
+                    for (int l = l0; l < p.natoms; l += 8) {
+                        cp_async_16(dst, src, src_bytes);
+                        dst += 1024u;
+                        src += 8 * plane_elems;
                     }
-                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                } else {
+                    for (int l = l0; l < p.natoms; l += 8, dst += 1024u)
+                        cp_async_16(dst, src_row + (int)ctl.atoms[l] * plane_elems, src_bytes);
                 }
-            }
-            PROF_STORE(0)
-            // drain: every load issued has either been consumed or is waited for here (bounded)
-            if (!ok) {
-                const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
-                for (uint32_t j = 0; j < n; ++j) {
-                    const uint32_t last = it - 1 - j;   // the most recent use of stage last % stages
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(&ctl.full[last % p.stages], (last / p.stages) & 1) && clock64() - t0 < (1ll << 27)) {}
-                }
+                // asynchronous arrival: counts on full[s] once this thread's copies above have landed
+                cp_async_mbar_arrive_noinc(&ctl.full[s]);
+                if (++s == p.stages) { s = 0; ph ^= 1; }
             }
         }
-        __syncwarp();
-    } else if (warp == 1) {
+        cp_async_wait_all();                                 // nothing of this thread is in flight at exit
+        PROF_STORE(warp)
+    } else if (warp == kMmaWarp) {
         // ===== MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_f16(128, G::NB, /*a_mn_major=*/true, /*b_mn_major=*/false);
@@ -328,8 +462,17 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_co
                 int f, y0, x0, rows;
                 decode_tile(p, t, f, y0, x0, rows);
                 for (int r = 0; r < rows; ++r, ++it) {
+#ifdef SR_PROFILE_ROLES
+                    if (debug_mode >= 1) {
+                        if (!(ok = mbar_wait(&ctl.full[s], ph, abort_flag))) break;
+                        mbar_arrive(&ctl.empty[s]);
+                        if (++s == p.stages) { s = 0; ph ^= 1; }
+                        continue;
+                    }
+#endif
                     if (!(ok = PROF_WAIT(mbar_wait(&ctl.acc_empty[a], aph ^ 1, abort_flag)))) break;
                     if (!(ok = PROF_WAIT(mbar_wait(&ctl.full[s], ph, abort_flag)))) break;
+                    fence_proxy_async_smem();        // the stage was written by cp.async (generic proxy), the MMA reads it through the async proxy
                     tc_fence_after_sync();
                     const uint32_t taddr = tmem_base + (uint32_t)(a * G::NB);
                     uint64_t ad = a_desc0 + (uint64_t)((uint32_t)s * a_stage_step);
@@ -349,8 +492,7 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_co
                     if (++a == G::ACC_SLOTS) { a = 0; aph ^= 1; }
                 }
             }
-            PROF_STORE(1)
-            PROF_STORE2(20, prof_mma, prof_commit)
+            PROF_STORE(warp)
         }
         __syncwarp();
     } else if (warp < kFirstEpiWarp) {
@@ -389,175 +531,169 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_all, const __grid_co
             bool ok = PROF_WAIT(mbar_wait(&ctl.u_empty[ub], uph ^ 1, abort_flag));
             ok = named_barrier_and(1, NU, ok);
             if (!ok) break;
+            PROF_T(tu0)
             if (has_next) prefetch_lr(t + gridDim.x, (ti + 1) & 1);
             const int uh = g.rows + 2 * G::P;
-            if (ut < G::UW) {
-                const int Xc = clampi(g.x0 - G::P + ut, 0, pb.W - 1);
-                const int q = fast_div(Xc, pb.r, p.r_magic), px = Xc - q * pb.r;
-                ctl.hx_off[ut] = q + pb.ph.base[px] - g.col_lo;
-                ctl.hx_w[ut] = make_float4(pb.ph.w[px][0], pb.ph.w[px][1], pb.ph.w[px][2], pb.ph.w[px][3]);
-            } else if (ut - G::UW < uh) {
-                const int uy = ut - G::UW;
-                const int Yc = clampi(g.y0 - G::P + uy, 0, pb.H - 1);
-                const int q = fast_div(Yc, pb.r, p.r_magic), py = Yc - q * pb.r;
-                ctl.vy_off[uy] = q + pb.ph.base[py] - g.lr_lo;
-                ctl.vy_w[uy] = make_float4(pb.ph.w[py][0], pb.ph.w[py][1], pb.ph.w[py][2], pb.ph.w[py][3]);
+            for (int i = ut; i < G::UW + uh; i += NU) {
+                if (i < G::UW) {
+                    const int Xc = clampi(g.x0 - G::P + i, 0, pb.W - 1);
+                    const int q = fast_div(Xc, pb.r, p.r_magic), px = Xc - q * pb.r;
+                    ctl.hx_off[i] = q + pb.ph.base[px] - g.col_lo;
+                    ctl.hx_w[i] = make_float4(pb.ph.w[px][0], pb.ph.w[px][1], pb.ph.w[px][2], pb.ph.w[px][3]);
+                } else {
+                    const int uy = i - G::UW;
+                    const int Yc = clampi(g.y0 - G::P + uy, 0, pb.H - 1);
+                    const int q = fast_div(Yc, pb.r, p.r_magic), py = Yc - q * pb.r;
+                    ctl.vy_off[uy] = q + pb.ph.base[py] - g.lr_lo;
+                    ctl.vy_w[uy] = make_float4(pb.ph.w[py][0], pb.ph.w[py][1], pb.ph.w[py][2], pb.ph.w[py][3]);
+                }
             }
             if (has_next) cp_async_wait<1>(); else cp_async_wait<0>();
             named_barrier_sync(1, NU);                       // tables written, this tile's LR window landed
-            // horizontal pass: T[row][ux] = sum_b wx[b] * L[row][hx_off[ux] + b], row = ch * nrows + j
+            PROF_ADD(prof_a, tu0)
+            PROF_T(tu1)
+            // horizontal pass: T[row][ux] = sum_b wx[b] * L[row][hx_off[ux] + b], row = ch * nrows + j;
+            // four neighbouring columns per trip, one 16-byte store
             const float* Lb = sL + (ti & 1) * lbuf_floats;
             const int hrows = C * g.nrows;
+            constexpr int UW4 = G::UW / 4;
 #pragma unroll 2
-            for (int o = ut; o < hrows * G::UW; o += NU) {
-                const int row = o / G::UW, ux = o - row * G::UW;
-                const float4 w = ctl.hx_w[ux];
-                const float* src = Lb + row * p.tcols + ctl.hx_off[ux];
-                float v = w.x * src[0];
-                v = fmaf(w.y, src[1], v);
-                v = fmaf(w.z, src[2], v);
-                v = fmaf(w.w, src[3], v);
-                sT[o] = v;
+            for (int o = ut; o < hrows * UW4; o += NU) {
+                const int row = o / UW4, ux = (o - row * UW4) * 4;
+                const int4 off = *reinterpret_cast<const int4*>(&ctl.hx_off[ux]);
+                const float* Lr = Lb + row * p.tcols;
+                float4 out;
+                {
+                    const float4 w = ctl.hx_w[ux];
+                    const float* src = Lr + off.x;
+                    out.x = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
+                }
+                {
+                    const float4 w = ctl.hx_w[ux + 1];
+                    const float* src = Lr + off.y;
+                    out.y = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
+                }
+                {
+                    const float4 w = ctl.hx_w[ux + 2];
+                    const float* src = Lr + off.z;
+                    out.z = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
+                }
+                {
+                    const float4 w = ctl.hx_w[ux + 3];
+                    const float* src = Lr + off.w;
+                    out.w = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
+                }
+                *reinterpret_cast<float4*>(sT + row * G::UW + ux) = out;
             }
+            PROF_ADD(prof_b, tu1)
+            PROF_T(tu2)
             named_barrier_sync(1, NU);
-            // vertical pass: U[ch][uy][ux] = sum_a wy[a] * T[ch * nrows + vy_off[uy] + a][ux]
+            PROF_ADD(prof_c, tu2)
+            PROF_T(tu3)
+            // vertical pass: U[ch][uy][ux] = sum_a wy[a] * T[ch * nrows + vy_off[uy] + a][ux], 16 bytes at a time
             float* Ub = sU + ub * C * G::UH * G::UW;
             for (int ch = 0; ch < C; ++ch) {
                 const float* Tc = sT + ch * g.nrows * G::UW;
                 float* Uc = Ub + ch * G::UH * G::UW;
 #pragma unroll 2
-                for (int o = ut; o < uh * G::UW; o += NU) {
-                    const int uy = o / G::UW, ux = o - uy * G::UW;
+                for (int o = ut; o < uh * UW4; o += NU) {
+                    const int uy = o / UW4, ux = (o - uy * UW4) * 4;
                     const float4 w = ctl.vy_w[uy];
                     const float* src = Tc + ctl.vy_off[uy] * G::UW + ux;
-                    float v = w.x * src[0];
-                    v = fmaf(w.y, src[G::UW], v);
-                    v = fmaf(w.z, src[2 * G::UW], v);
-                    v = fmaf(w.w, src[3 * G::UW], v);
-                    Uc[o] = v;
+                    const float4 t0 = *reinterpret_cast<const float4*>(src);
+                    const float4 t1 = *reinterpret_cast<const float4*>(src + G::UW);
+                    const float4 t2 = *reinterpret_cast<const float4*>(src + 2 * G::UW);
+                    const float4 t3 = *reinterpret_cast<const float4*>(src + 3 * G::UW);
+                    float4 out;
+                    out.x = fmaf(w.w, t3.x, fmaf(w.z, t2.x, fmaf(w.y, t1.x, w.x * t0.x)));
+                    out.y = fmaf(w.w, t3.y, fmaf(w.z, t2.y, fmaf(w.y, t1.y, w.x * t0.y)));
+                    out.z = fmaf(w.w, t3.z, fmaf(w.z, t2.z, fmaf(w.y, t1.z, w.x * t0.z)));
+                    out.w = fmaf(w.w, t3.w, fmaf(w.z, t2.w, fmaf(w.y, t1.w, w.x * t0.w)));
+                    *reinterpret_cast<float4*>(Uc + uy * G::UW + ux) = out;
                 }
             }
+            PROF_ADD(prof_d, tu3)
             mbar_arrive(&ctl.u_full[ub]);
         }
         cp_async_wait<0>();
         PROF_STORE(warp)
     } else {
-        // ===== epilogue: thread = one pixel column of the tile (TMEM lane), rows in order
-        const int quarter = warp & 3;                        // the TMEM lanes this warp may read: 32*quarter..+31
-        const int x = quarter * 32 + lane;                   // pixel within the tile row
-        const int64_t HW = (int64_t)pb.H * pb.W;
-        const bool clamp01 = (pb.flags & SR_CLAMP01) != 0;
-        uint32_t it = 0, ti = 0;
+        // ===== epilogue: thread = one pixel column of the tile (TMEM lane); two groups of four warps own the
+        // upper and the lower half of a tile and walk their rows top to bottom
+        EpiCtx e;
+        e.quarter = warp & 3;                                // the TMEM lanes this warp may read: 32*quarter..+31
+        e.group = (warp - kFirstEpiWarp) >> 2;
+        e.x = e.quarter * 32 + lane;                         // pixel within the tile row
+        e.HW = (int64_t)pb.H * pb.W;
+        e.clamp01 = (pb.flags & SR_CLAMP01) != 0;
+        e.tmem_lane_base = tmem_base + ((uint32_t)(e.quarter * 32) << 16);
+        uint32_t it_base = 0, ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++ti) {
             int f, y0, x0, rows;
             decode_tile(p, t, f, y0, x0, rows);
             const int ub = ti & 1;
             const uint32_t uph = (ti >> 1) & 1;
-            ok = PROF_WAIT(__all_sync(0xffffffffu, mbar_wait(&ctl.u_full[ub], uph, abort_flag)));
+            ok = PROF_WAIT(mbar_wait_warp(&ctl.u_full[ub], uph, abort_flag));
             if (!ok) break;
-            const float* Ub = sU + ub * C * G::UH * G::UW;
-            const bool in_x = x0 + x < pb.W;
-            float* dst0 = p.out + ((int64_t)f * C) * HW + (int64_t)y0 * pb.W + x0 + x;
+            const int h1 = rows > kHalf ? rows - kHalf : 0;
+            const int my_rows = e.group ? h1 : rows - h1;    // rows of this group's half
+            const int r0 = e.group * kHalf;                  // first tile row of the half
+            const float* Ub = sU + ub * C * G::UH * G::UW + r0 * G::UW;
+            const bool in_x = x0 + e.x < pb.W;
+            float* dst0 = p.out + ((int64_t)f * C) * e.HW + (int64_t)(y0 + r0) * pb.W + x0 + e.x;
             if (K <= 5 && C == 3) {
-                // sliding window: the k x k x 3 patch lives in registers; each new row costs 3k shared loads
-                float win[3][K][K];
-                const float* u0 = Ub + x;
-#pragma unroll
-                for (int a = 0; a < K - 1; ++a)
-#pragma unroll
-                    for (int c = 0; c < 3; ++c)
-#pragma unroll
-                        for (int b = 0; b < K; ++b) win[c][a][b] = u0[(c * G::UH + a) * G::UW + b];
-#pragma unroll
-                for (int r = 0; r < TH; ++r) {
-                    if (r < rows && ok) {
-#pragma unroll
-                        for (int c = 0; c < 3; ++c)
-#pragma unroll
-                            for (int b = 0; b < K; ++b) win[c][(r + K - 1) % K][b] = u0[(c * G::UH + r + K - 1) * G::UW + b];
-                        const int a_slot = it % G::ACC_SLOTS;
-                        const uint32_t aph = (it / G::ACC_SLOTS) & 1;
-                        ok = PROF_WAIT(__all_sync(0xffffffffu, mbar_wait(&ctl.acc_full[a_slot], aph, abort_flag)));
-                        if (ok) {
-                            tc_fence_after_sync();
-                            float F[G::NPAD];
-                            load_filter<K>(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a_slot * G::NB), F);
-                            tc_fence_before_sync();
-                            mbar_arrive(&ctl.acc_empty[a_slot]);
-                            float acc[3][2];
-#pragma unroll
-                            for (int c = 0; c < 3; ++c) acc[c][0] = acc[c][1] = 0.f;
-#pragma unroll
-                            for (int a = 0; a < K; ++a)
-#pragma unroll
-                                for (int b = 0; b < K; ++b)
-#pragma unroll
-                                    for (int c = 0; c < 3; ++c)
-                                        acc[c][a & 1] = fmaf(F[a * K + b], win[c][(r + a) % K][b], acc[c][a & 1]);
-#pragma unroll
-                            for (int c = 0; c < 3; ++c) {
-                                float v = acc[c][0] + acc[c][1];
-                                if (clamp01) v = fminf(fmaxf(v, 0.f), 1.f);
-                                if (in_x) dst0[c * HW + (int64_t)r * pb.W] = v;
-                            }
-                        }
-                        ++it;
-                    }
-                }
+                ok = epilogue_half_windowed<K>(ctl, e, Ub, dst0, pb.W, my_rows, h1, it_base, in_x, abort_flag);
             } else {
-                for (int r = 0; r < rows; ++r, ++it) {
+                for (int j = 0; j < my_rows; ++j) {
+                    const uint32_t it = it_base + item_of_half_row(j, e.group, h1);
                     const int a_slot = it % G::ACC_SLOTS;
                     const uint32_t aph = (it / G::ACC_SLOTS) & 1;
-                    ok = PROF_WAIT(__all_sync(0xffffffffu, mbar_wait(&ctl.acc_full[a_slot], aph, abort_flag)));
+                    ok = mbar_wait_warp(&ctl.acc_full[a_slot], aph, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
                     float F[G::NPAD];
-                    load_filter<K>(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a_slot * G::NB), F);
+                    load_filter<K>(e.tmem_lane_base + (uint32_t)(a_slot * G::NB), F);
                     tc_fence_before_sync();
                     mbar_arrive(&ctl.acc_empty[a_slot]);
-                    float* dst = dst0 + (int64_t)r * pb.W;
-                    const float* u0 = Ub + r * G::UW + x;
+                    float* dst = dst0 + (int64_t)j * pb.W;
+                    const float* u0 = Ub + j * G::UW + e.x;
                     if (C == 3) {
-                        patch_dot<K, 3>(F, u0, G::UH * G::UW, G::UW, dst, HW, in_x, clamp01);
+                        patch_dot<K, 3>(F, u0, G::UH * G::UW, G::UW, dst, e.HW, in_x, e.clamp01);
                     } else {
                         for (int ch = 0; ch < C; ++ch)
-                            patch_dot<K, 1>(F, u0 + ch * G::UH * G::UW, G::UH * G::UW, G::UW, dst + ch * HW, HW, in_x, clamp01);
+                            patch_dot<K, 1>(F, u0 + ch * G::UH * G::UW, G::UH * G::UW, G::UW, dst + ch * e.HW, e.HW, in_x, e.clamp01);
                     }
                 }
             }
+            it_base += rows;
             if (ok) mbar_arrive(&ctl.u_empty[ub]);
         }
         PROF_STORE(warp)
     }
 
     // ---------------------------------------------------------------- teardown
+#ifdef SR_PROFILE_ROLES
+teardown:
+#endif
     __syncwarp();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+#ifdef SR_PROFILE_ROLES
+    if (tid == 0 && g_role_prof) {
+        unsigned long long gt_end; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_end));
+        g_role_prof[(blockIdx.x * 32 + 30) * 2] = (long long)(gt_setup - gt_entry);
+        g_role_prof[(blockIdx.x * 32 + 30) * 2 + 1] = (long long)(gt_end - gt_entry);
+        g_role_prof[(blockIdx.x * 32 + 31) * 2] = (long long)gt_entry;
+        g_role_prof[(blockIdx.x * 32 + 31) * 2 + 1] = (long long)gt_end;
+    }
+#endif
     if (ctl.abort_flag && tid == 0) atomicExch(p.status, SR_ERR_TIMEOUT);
-    if (warp == 1) tmem_dealloc(tmem_base, G::TMEM_COLS);
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, G::TMEM_COLS);
 }
 
 // ---- host side -------------------------------------------------------------------------------------------------------
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            f = nullptr;
-        return (EncodeTiledFn)f;
-    }();
-    return fn;
-}
 
 struct DeviceInfo { int sms = 0, cc_major = 0, smem_optin = 0; bool ok = false; };
 
@@ -578,7 +714,7 @@ const DeviceInfo& device_info()
 }
 
 int trows_for(int k, int r) { return (TH + (k - 1) - 1) / r + 5; }
-int tcols_for(int k, int r) { return (TW + (k - 1) - 1) / r + 5; }
+int tcols_for(int k, int r) { return (((TW + (k - 1) + 3) & ~3) - 1) / r + 5; }
 
 template <int K> size_t fixed_smem_bytes(int c, int dpad, int r)
 {
@@ -589,14 +725,14 @@ template <int K> size_t fixed_smem_bytes(int c, int dpad, int r)
 }
 
 // planes that enter the contraction, and whether they are picked one by one out of a full tensor
-void contraction_shape(int mode, const Problem& pb, int& natoms, int& per_atom)
+void contraction_shape(int mode, const Problem& pb, int& natoms, int& gather)
 {
     if (mode == kModeGlobal) {
         natoms = pb.s;
-        per_atom = (pb.flags & SR_COEF_COMPACT) ? 0 : 1;
+        gather = (pb.flags & SR_COEF_COMPACT) ? 0 : 1;
     } else {
         natoms = pb.D;
-        per_atom = 0;
+        gather = 0;
     }
 }
 
@@ -620,7 +756,7 @@ int stages_for_k(int k, int c, int dpad, int r, int smem_optin)
 }
 
 template <int K>
-cudaError_t launch_k(const CUtensorMap& map_all, const CUtensorMap& map_row, UmmaParams& prm, cudaStream_t st)
+cudaError_t launch_k(UmmaParams& prm, cudaStream_t st)
 {
     const DeviceInfo& di = device_info();
     const size_t smem = fixed_smem_bytes<K>(prm.pb.c, prm.dpad, prm.pb.r) + (size_t)prm.stages * prm.dpad * 256;
@@ -634,7 +770,7 @@ cudaError_t launch_k(const CUtensorMap& map_all, const CUtensorMap& map_row, Umm
         configured[dev] = true;
     }
     const int grid = prm.num_tiles < di.sms ? prm.num_tiles : di.sms;
-    kern<<<grid, kThreads, smem, st>>>(map_all, map_row, prm);
+    kern<<<grid, kThreads, smem, st>>>(prm);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -642,6 +778,11 @@ cudaError_t launch_k(const CUtensorMap& map_all, const CUtensorMap& map_row, Umm
 } // namespace
 
 #ifdef SR_PROFILE_ROLES
+extern "C" int sr_debug_mode(int mode)
+{
+    return cudaMemcpyToSymbol(g_debug_mode, &mode, sizeof(mode)) == cudaSuccess ? 0 : 5;
+}
+
 extern "C" int sr_debug_role_profile(long long* device_buffer)
 {
     return cudaMemcpyToSymbol(g_role_prof, &device_buffer, sizeof(device_buffer)) == cudaSuccess ? 0 : 5;
@@ -653,12 +794,12 @@ bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& p
     if (mode != kModeDense && mode != kModeGlobal) return false;
     if (coef_dtype != SR_F16) return false;
     if (pb.k > 7 || pb.c > kMaxChannels) return false;
-    if ((reinterpret_cast<uintptr_t>(coef) & 15) != 0 || (pb.W & 7) != 0) return false;   // TMA: 16-byte base and pitches
+    if ((reinterpret_cast<uintptr_t>(coef) & 15) != 0 || (pb.W & 7) != 0) return false;   // 16-byte copies: aligned base and row pitch
     if (pb.n > 65535) return false;
     const DeviceInfo& di = device_info();
-    if (!di.ok || di.cc_major != 10 || !encode_fn()) return false;
-    int natoms, per_atom;
-    contraction_shape(mode, pb, natoms, per_atom);
+    if (!di.ok || di.cc_major != 10) return false;
+    int natoms, gather;
+    contraction_shape(mode, pb, natoms, gather);
     const int dpad = (natoms + 15) / 16 * 16;
     return stages_for_k(pb.k, pb.c, dpad, pb.r, di.smem_optin) >= 2;
 }
@@ -673,7 +814,9 @@ cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, con
     if (!prm.status) return cudaErrorUnknown;
     prm.pb = pb;
     prm.mode = mode;
-    contraction_shape(mode, pb, prm.natoms, prm.per_atom_boxes);
+    contraction_shape(mode, pb, prm.natoms, prm.gather_planes);
+    prm.planes = (mode == kModeGlobal && (pb.flags & SR_COEF_COMPACT)) ? pb.s : pb.D;
+    prm.coef = static_cast<const __half*>(coef);
     prm.dpad = (prm.natoms + 15) / 16 * 16;
     prm.stages = stages_for_k(pb.k, pb.c, prm.dpad, pb.r, di.smem_optin);
     prm.trows = trows_for(pb.k, pb.r);
@@ -684,29 +827,11 @@ cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, con
     prm.tiles_y = (pb.H + TH - 1) / TH;
     prm.num_tiles = prm.tiles_x * prm.tiles_y * pb.n;
 
-    // coefficient tensor as seen by TMA: (W, H, planes, n) binary16, innermost first
-    const int planes = (mode == kModeGlobal && (pb.flags & SR_COEF_COMPACT)) ? pb.s : pb.D;
-    const cuuint64_t dims[4] = {(cuuint64_t)pb.W, (cuuint64_t)pb.H, (cuuint64_t)planes, (cuuint64_t)pb.n};
-    const cuuint64_t strides[3] = {(cuuint64_t)pb.W * 2, (cuuint64_t)pb.W * pb.H * 2, (cuuint64_t)pb.W * pb.H * 2 * planes};
-    const cuuint32_t es[4] = {1, 1, 1, 1};
-    const cuuint32_t box_all[4] = {64, 1, (cuuint32_t)prm.dpad, 1};
-    const cuuint32_t box_row[4] = {64, 1, 1, 1};
-    CUtensorMap map_all, map_row;
-    EncodeTiledFn enc = encode_fn();
-    if (enc(&map_all, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(coef), dims, strides, box_all, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
-    if (enc(&map_row, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(coef), dims, strides, box_row, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
-
     switch (pb.k) {
-    case 1: return launch_k<1>(map_all, map_row, prm, st);
-    case 3: return launch_k<3>(map_all, map_row, prm, st);
-    case 5: return launch_k<5>(map_all, map_row, prm, st);
-    case 7: return launch_k<7>(map_all, map_row, prm, st);
+    case 1: return launch_k<1>(prm, st);
+    case 3: return launch_k<3>(prm, st);
+    case 5: return launch_k<5>(prm, st);
+    case 7: return launch_k<7>(prm, st);
     default: return cudaErrorNotSupported;
     }
 }
