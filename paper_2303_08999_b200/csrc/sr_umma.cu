@@ -16,13 +16,17 @@
 // Shared-memory bandwidth and per-warp latency are the scarce on-chip resources, so the epilogue keeps a sliding
 // k x k x 3 window of U in registers and reads each U row once per pixel column.
 //
-// Warp roles (512 threads):
+// Warp roles (640 threads = five warpgroups; the register file is re-balanced between them with setmaxnreg):
 //   warps 0-3    coefficient producers   full[stage] <- cp.async arrivals when the copies land; wait empty[stage]
-//   warp 4       MMA issuer, TMEM owner  acc_full[a], empty[stage] <- tcgen05.commit; waits full[stage], acc_empty[a]
-//   warps 5-7    U producers             bicubic (separable) of the tile + halo into a double-buffered tile
-//   warps 8-15   epilogue (2 x 4 warps)  TMEM -> registers (one pixel's filter per thread), patch dot, clamp, store;
+//   warps 4-5    MMA issuers (warp 4 owns TMEM): one thread each, alternate rows, because the issue loop of a
+//                single thread (~600 cycles per row alone, twice that on a busy SM) would otherwise pace the kernel;
+//                acc_full[a], empty[stage] <- tcgen05.commit; wait full[stage], acc_empty[a]
+//   warps 6-11   U producers             bicubic (separable) of the tile + halo into a double-buffered tile
+//   warps 12-19  epilogue (2 x 4 warps)  TMEM -> registers (one pixel's filter per thread), patch dot, clamp, store;
 //                                        the two groups own the upper and the lower half of a tile
 // Every wait is bounded; on expiry the CTA raises its abort flag, sets the device status word and drains.
+#include <stdlib.h>
+
 #include "sr_ptx.cuh"
 #include "sr_umma.cuh"
 
@@ -33,10 +37,14 @@ namespace {
 using namespace ptx;
 
 constexpr int TW = 128, TH = 16;
-constexpr int kThreads = 512;
-constexpr int kNumLoadWarps = 4, kMmaWarp = 4;
-constexpr int kFirstUWarp = 5, kNumUWarps = 3, kFirstEpiWarp = 8, kNumEpiWarps = 8;
-constexpr int kMaxStages = 8;
+constexpr int kThreads = 640;
+constexpr int kNumLoadWarps = 4, kMmaWarp = 4, kNumMmaWarps = 2;
+constexpr int kFirstUWarp = 6, kNumUWarps = 6, kFirstEpiWarp = 12, kNumEpiWarps = 8;
+// Registers per thread after the warpgroups re-balance the register file (setmaxnreg): 20 warps start at 96;
+// loaders and the MMA / U warpgroups give registers back, the two epilogue warpgroups take them.
+// 4*40 + 8*72 + 8*144 = 1888 <= 2048 warp-registers.
+constexpr int kRegsLoad = 40, kRegsMmaU = 72, kRegsEpi = 144;
+constexpr int kMaxStages = 10;
 constexpr int kMaxAccSlots = 8;
 constexpr int kMaxChannels = 4;
 constexpr int kStaticReserve = 5120;   // static shared memory (control block) + alignment, kept out of the dynamic budget
@@ -52,7 +60,12 @@ struct UmmaParams {
     int mode;
     int natoms;           // coefficient planes per pixel that enter the contraction (D, or s for a subset)
     int dpad;             // natoms rounded up to a multiple of 16 (the MMA K extent)
+    int rows_alloc;       // rows a stage chunk really holds: natoms rounded up to 8 (one swizzle group). When this is
+                          // below dpad the last K-step's upper 8 rows read whatever follows the chunk; the matching
+                          // dictionary rows are zero, so any finite bytes there contribute nothing.
     int planes;           // planes per frame in the coefficient tensor (D, or s when it is compact)
+    int tma_rows;         // leading planes of every stage that a TMA box brings in (multiple of 8; 0 = none); the
+                          // rest arrive through cp.async, so that both load paths of the SM work side by side
     int gather_planes;    // 1: plane q of the contraction is plane atoms[q] of the tensor (subset of a full tensor)
     const __half* coef;
     int stages;
@@ -70,9 +83,9 @@ struct __align__(16) Ctl {
     uint32_t tmem_base;
     int abort_flag;
     float4 vy_w[TH + 2 * 4];   // per U-tile row: its four vertical tap weights
-    float4 hx_w[TW + 2 * 4];   // per U-tile column: its four horizontal tap weights
+    float4 wtab[kMaxScale];    // the four tap weights of every phase (copied once from the kernel parameters)
     int vy_off[TH + 2 * 4];    // per U-tile row: first row of the scratch tile it reads
-    alignas(16) int hx_off[TW + 2 * 4];   // per U-tile column: first column of the LR window it reads
+    alignas(16) int hx_off[TW + 2 * 4];   // per U-tile column: first column of the LR window it reads, | phase << 16
     uint8_t atoms[256];        // subset mode: the atom id of each selected plane
 };
 
@@ -86,6 +99,12 @@ template <int K> struct Geo {
     static constexpr int LBO_B = (NB / 8) * 128;         // bytes between the two K-halves of a K-step of the B operand
     static constexpr int KSTEP_B = 2 * LBO_B;            // bytes per K-step (16 atoms) of the B operand
     static constexpr int ACC_SLOTS = (512 / NB) < kMaxAccSlots ? (512 / NB) : kMaxAccSlots;
+    // Column of tap (a, b) inside a half of the accumulator: the first K-1 taps of every patch row come first, row by
+    // row, so that they can be consumed as aligned pairs by the packed fp32 instructions; the last tap of every row
+    // follows as a block of K single columns.
+    static constexpr int NPAIRCOLS = K * (K - 1);
+    __host__ __device__ static constexpr int col_of(int a, int b) { return b < K - 1 ? a * (K - 1) + b : NPAIRCOLS + a; }
+    __host__ __device__ static constexpr int col_of_tap(int j) { return col_of(j / K, j % K); }
     static constexpr int TMEM_COLS = ACC_SLOTS * NB;     // 256 or 512: a power of two
 };
 
@@ -137,6 +156,9 @@ __device__ __forceinline__ void cp_async_f32(float* dst_smem, const float* src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
 }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 // 16-byte copy global -> shared, L1 bypassed; src_bytes = 0 writes zeros instead of reading.
 __device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src, uint32_t src_bytes)
 {
@@ -183,11 +205,13 @@ __device__ __forceinline__ bool named_barrier_and(int id, int nthreads, bool pre
     return r != 0;
 }
 
-// One pixel's filter from tensor memory: F[j] = hi[j] + lo[j] for the taps j < k*k (at most 16 columns at a time).
+// One pixel's filter from tensor memory in natural tap order: F[a*K+b] = hi[col] + lo[col], col = col_of(a, b)
+// (at most 16 columns at a time).
 template <int K>
 __device__ __forceinline__ void load_filter(uint32_t taddr, float* F)
 {
     using G = Geo<K>;
+    float Fc[G::NPAD];                                       // column order
 #pragma unroll
     for (int j0 = 0; j0 < G::kk; j0 += 16) {
         constexpr int kTail = G::kk % 16;
@@ -202,8 +226,10 @@ __device__ __forceinline__ void load_filter(uint32_t taddr, float* F)
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-            if (j0 + i < G::kk) F[j0 + i] = h[i] + l[i];
+            if (j0 + i < G::kk) Fc[j0 + i] = h[i] + l[i];
     }
+#pragma unroll
+    for (int j = 0; j < G::kk; ++j) F[j] = Fc[G::col_of_tap(j)];
 }
 
 // y_c = F . B_c for NC channels of one pixel, patch read tap by tap from the shared U tile. Independent
@@ -242,55 +268,92 @@ __device__ __forceinline__ int item_of_half_row(int j, int group, int h1)
     return j < h1 ? 2 * j + group : j + h1;              // beyond h1 only the upper half (group 0) has rows
 }
 
-// Epilogue of one half tile (rows j = 0 .. my_rows-1 of the half, top to bottom) for a three-channel image:
-// the k x k x 3 patch lives in registers as a sliding window (slot of U row u is u % K, all indices
-// compile-time), so each row costs 3 * K shared loads instead of 3 * K * K. Returns false when a wait expired.
+// Epilogue of one half tile (rows j = 0 .. my_rows-1 of the half, top to bottom) for a three-channel image.
+// The k x k x 3 patch lives in registers as a sliding window (slot of U row u is u % K, all indices
+// compile-time), so each row costs 3 * K shared loads instead of 3 * K * K. Window rows and filter taps are held
+// as (K-1)/2 aligned pairs plus one single per patch row, so hi + lo and the patch dot product run on the packed
+// fp32 instructions (two lanes per issue slot). Returns false when a wait expired.
 template <int K, class CtlT>
 __device__ __forceinline__ bool epilogue_half_windowed(CtlT& ctl, const EpiCtx& e, const float* Ub, float* dst0, int W,
                                                        int my_rows, int h1, uint32_t it_base, bool in_x,
-                                                       volatile int* abort_flag)
+                                                       volatile int* abort_flag, long long* wait_cycles = nullptr)
 {
     using G = Geo<K>;
-    float win[3][K][K];
+    constexpr int NP = (K - 1) / 2;                          // pairs per patch row
+    constexpr int NPc = NP > 0 ? NP : 1;
+    float2 winp[3][K][NPc];
+    float wins[3][K];
     const float* u0 = Ub + e.x;
+    auto load_row = [&](int u) {                             // U row u of the half -> window slot u % K
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            const float* src = u0 + (c * G::UH + u) * G::UW;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) winp[c][u % K][i] = make_float2(src[2 * i], src[2 * i + 1]);
+            wins[c][u % K] = src[K - 1];
+        }
+    };
     bool ok = true;
     if (my_rows > 0) {
 #pragma unroll
-        for (int u = 0; u < K - 1; ++u)
-#pragma unroll
-            for (int c = 0; c < 3; ++c)
-#pragma unroll
-                for (int b = 0; b < K; ++b) win[c][u][b] = u0[(c * G::UH + u) * G::UW + b];
+        for (int u = 0; u < K - 1; ++u) load_row(u);
     }
 #pragma unroll
     for (int j = 0; j < kHalf; ++j) {
         if (j < my_rows && ok) {
-#pragma unroll
-            for (int c = 0; c < 3; ++c)
-#pragma unroll
-                for (int b = 0; b < K; ++b) win[c][(j + K - 1) % K][b] = u0[(c * G::UH + j + K - 1) * G::UW + b];
+            load_row(j + K - 1);
             const uint32_t it = it_base + item_of_half_row(j, e.group, h1);
             const int a_slot = it % G::ACC_SLOTS;
             const uint32_t aph = (it / G::ACC_SLOTS) & 1;
+#ifdef SR_PROFILE_ROLES
+            const long long tw0 = clock64();
+#endif
             ok = mbar_wait_warp(&ctl.acc_full[a_slot], aph, abort_flag);
+#ifdef SR_PROFILE_ROLES
+            if (wait_cycles) *wait_cycles += clock64() - tw0;
+#endif
             if (ok) {
                 tc_fence_after_sync();
-                float F[G::NPAD];
-                load_filter<K>(e.tmem_lane_base + (uint32_t)(a_slot * G::NB), F);
+                const uint32_t taddr = e.tmem_lane_base + (uint32_t)(a_slot * G::NB);
+                // filter: pair columns [0, K(K-1)) and single columns [K(K-1), K*K) of both halves, summed
+                float2 Fp[K][NPc];
+                float Fs[K];
+                {
+                    float2 hp[K * NPc], lp[K * NPc];
+                    if (NP > 0) {
+                        tmem_ld_n<G::NPAIRCOLS>(taddr, reinterpret_cast<float*>(hp));
+                        tmem_ld_n<G::NPAIRCOLS>(taddr + G::NPAD, reinterpret_cast<float*>(lp));
+                    }
+                    float hs[K], ls[K];
+                    tmem_ld_n<K>(taddr + G::NPAIRCOLS, hs);
+                    tmem_ld_n<K>(taddr + G::NPAD + G::NPAIRCOLS, ls);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int a = 0; a < K; ++a) {
+#pragma unroll
+                        for (int i = 0; i < NP; ++i) Fp[a][i] = __fadd2_rn(hp[a * NP + i], lp[a * NP + i]);
+                        Fs[a] = hs[a] + ls[a];
+                    }
+                }
                 tc_fence_before_sync();
                 mbar_arrive(&ctl.acc_empty[a_slot]);
-                float acc[3][2];
+                float2 acc2[3][2];
+                float accs[3];
 #pragma unroll
-                for (int c = 0; c < 3; ++c) acc[c][0] = acc[c][1] = 0.f;
+                for (int c = 0; c < 3; ++c) { acc2[c][0] = acc2[c][1] = make_float2(0.f, 0.f); accs[c] = 0.f; }
 #pragma unroll
                 for (int a = 0; a < K; ++a)
 #pragma unroll
-                    for (int b = 0; b < K; ++b)
+                    for (int c = 0; c < 3; ++c) {
 #pragma unroll
-                        for (int c = 0; c < 3; ++c) acc[c][a & 1] = fmaf(F[a * K + b], win[c][(j + a) % K][b], acc[c][a & 1]);
+                        for (int i = 0; i < NP; ++i)
+                            acc2[c][i & 1] = __ffma2_rn(Fp[a][i], winp[c][(j + a) % K][i], acc2[c][i & 1]);
+                        accs[c] = fmaf(Fs[a], wins[c][(j + a) % K], accs[c]);
+                    }
 #pragma unroll
                 for (int c = 0; c < 3; ++c) {
-                    float v = acc[c][0] + acc[c][1];
+                    const float2 t2 = __fadd2_rn(acc2[c][0], acc2[c][1]);
+                    float v = (t2.x + t2.y) + accs[c];
                     if (e.clamp01) v = fminf(fmaxf(v, 0.f), 1.f);
                     if (in_x) dst0[c * e.HW + (int64_t)j * W] = v;
                 }
@@ -322,7 +385,7 @@ __device__ int g_debug_mode = 0;   // 1: TMA streaming only (no MMA, no U, no ep
 
 template <int K>
 __global__ void __launch_bounds__(kThreads, 1)
-regress_umma_kernel(const __grid_constant__ UmmaParams p)
+regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_constant__ UmmaParams p)
 {
     using G = Geo<K>;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -334,8 +397,8 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
 #endif
     const Problem& pb = p.pb;
     const int C = pb.c;
-    const int stage_bytes = p.dpad * 256;            // two chunks of [dpad][64 pixels] binary16
-    const int chunk_bytes = p.dpad * 128;
+    const int stage_bytes = p.rows_alloc * 256;      // two chunks of [rows_alloc][64 pixels] binary16
+    const int chunk_bytes = p.rows_alloc * 128;
     const int ksteps = p.dpad / 16;
 
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -347,11 +410,12 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
-        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], kNumLoadWarps * 32); mbar_init(&ctl.empty[i], 1); }
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], kNumLoadWarps * 32 + (p.tma_rows > 0 ? 1 : 0)); mbar_init(&ctl.empty[i], 1); }
         for (int i = 0; i < kMaxAccSlots; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], 128); }
         for (int i = 0; i < 2; ++i) { mbar_init(&ctl.u_full[i], kNumUWarps * 32); mbar_init(&ctl.u_empty[i], kNumEpiWarps * 32); }
         ctl.abort_flag = 0;
         fence_barrier_init();
+        if (p.tma_rows > 0) prefetch_tensormap(&map_lead);
     }
     // B operand: dict (or gamma-weighted subset rows) as binary16 hi | lo along N, K-major, no swizzle.
     // element (column n, atom k) of a K-step: (k%16)/8 * LBO + n/8 * 128 + n%8 * 16 + k%8 * 2
@@ -369,10 +433,12 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
         const __half hi = __float2half_rn(v);
         const __half lo = __float2half_rn(v - __half2float(hi));
         const int base = (k >> 4) * G::KSTEP_B + ((k & 15) >> 3) * G::LBO_B + (k & 7) * 2;
-        const int nl = n + G::NPAD;
-        *reinterpret_cast<__half*>(sB + base + (n >> 3) * 128 + (n & 7) * 16) = hi;
+        const int nh = n < G::kk ? G::col_of_tap(n) : n;     // tap n lives in column col_of_tap(n) of each half
+        const int nl = nh + G::NPAD;
+        *reinterpret_cast<__half*>(sB + base + (nh >> 3) * 128 + (nh & 7) * 16) = hi;
         *reinterpret_cast<__half*>(sB + base + (nl >> 3) * 128 + (nl & 7) * 16) = lo;
     }
+    if (tid < kMaxScale) ctl.wtab[tid] = make_float4(pb.ph.w[tid][0], pb.ph.w[tid][1], pb.ph.w[tid][2], pb.ph.w[tid][3]);
     if (p.gather_planes)
         for (int q = tid; q < p.natoms; q += kThreads) ctl.atoms[q] = (uint8_t)min((int)__ldg(p.idx + q), pb.D - 1);
     // The copies only ever write rows < natoms of a stage; the padding rows up to dpad must read as zero.
@@ -397,9 +463,16 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
     // ---------------------------------------------------------------- roles
 #ifdef SR_PROFILE_ROLES
     const int debug_mode = g_debug_mode;
-    if (debug_mode >= 1 && warp > kMmaWarp) goto teardown;
+    // debug runs: 1, 2 = streaming only; 3 = loaders + MMA + epilogue handshake only (no U, no TMEM reads, no math)
+    const int dm = debug_mode & 15;
+    const int my_tiles = ((dm == 1 || dm == 2) && warp > kMmaWarp) || ((dm >= 3 && dm <= 5) && warp > kMmaWarp && warp < kFirstEpiWarp) ? 0 : p.num_tiles;
+#else
+    const int my_tiles = p.num_tiles;
 #endif
+    // Each role's branch starts by re-balancing the register file for its warpgroup (all four warps of a
+    // warpgroup execute the same setmaxnreg instruction).
     if (warp < kNumLoadWarps) {
+        setmaxnreg_dec<kRegsLoad>();
         // ===== coefficient producers: 128 threads, thread = (16-byte column c16 of the 128-pixel row, atom l0 + 8k)
         // A stage is [chunk of 64 pixels][atom][128 B]; within a 1024-byte group of 8 atoms the 16-byte columns are
         // XOR-swizzled with the atom index (the 128-byte swizzle the MMA descriptor names).
@@ -414,21 +487,30 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
             int f, y0, x0, rows;
             decode_tile(p, t, f, y0, x0, rows);
 #ifdef SR_PROFILE_ROLES
-            if (debug_mode == 2) { int rr; decode_tile(p, blockIdx.x % p.tiles_x, f, y0, x0, rr); }   // L2-resident re-reads
+            if ((debug_mode & 15) == 2) { int rr; decode_tile(p, blockIdx.x % p.tiles_x, f, y0, x0, rr); }   // L2-resident re-reads
 #endif
             const int xe = x0 + c16 * 8;                     // first of this thread's 8 pixels
             const uint32_t src_bytes = xe < pb.W ? 16u : 0u; // columns beyond the image are zero-filled
             const __half* src_col = p.coef + (int64_t)f * p.planes * plane_elems + (xe < pb.W ? xe : 0);
             for (int r = 0; r < rows; ++r) {
-                ok = PROF_WAIT(mbar_wait_warp(&ctl.empty[s], ph ^ 1, abort_flag));
+                ok = PROF_WAIT(mbar_wait(&ctl.empty[s], ph ^ 1, abort_flag));
                 if (!ok) break;
                 const int yr = y0 + tile_row_of_item(r, rows);
                 const __half* src_row = src_col + (int64_t)yr * pb.W;
                 uint32_t dst = smem_u32(sA + (size_t)s * stage_bytes) + dst_thread;
+                if (p.tma_rows > 0 && tid == 0) {
+                    // planes [0, tma_rows) of both 64-pixel chunks: two boxes, bytes counted on the same barrier
+                    uint8_t* sdst = sA + (size_t)s * stage_bytes;
+                    mbar_arrive_expect_tx(&ctl.full[s], (uint32_t)p.tma_rows * 256u);
+                    tma_load_4d(sdst, &map_lead, &ctl.full[s], x0, yr, 0, f);
+                    tma_load_4d(sdst + chunk_bytes, &map_lead, &ctl.full[s], x0 + 64, yr, 0, f);
+                }
                 if (!p.gather_planes) {
-                    const __half* src = src_row + l0 * plane_elems;
+                    const int lfirst = p.tma_rows + l0;
+                    const __half* src = src_row + lfirst * plane_elems;
+                    dst += (uint32_t)p.tma_rows * 128u;
 #pragma unroll 3
-                    for (int l = l0; l < p.natoms; l += 8) {
+                    for (int l = lfirst; l < p.natoms; l += 8) {
                         cp_async_16(dst, src, src_bytes);
                         dst += 1024u;
                         src += 8 * plane_elems;
@@ -444,8 +526,10 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
         }
         cp_async_wait_all();                                 // nothing of this thread is in flight at exit
         PROF_STORE(warp)
-    } else if (warp == kMmaWarp) {
-        // ===== MMA issuer
+    } else if (warp < kFirstEpiWarp) {
+      setmaxnreg_dec<kRegsMmaU>();
+      if (warp < kMmaWarp + kNumMmaWarps) {
+        // ===== MMA issuers: warp kMmaWarp + m takes the rows whose running index is m modulo kNumMmaWarps
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_f16(128, G::NB, /*a_mn_major=*/true, /*b_mn_major=*/false);
             // A: MN-major, 128-byte swizzle: 8 atoms x 64 pixels per 1024-byte atom; K-groups 1024 B apart (SBO),
@@ -454,48 +538,47 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
             const uint64_t a_desc0 = make_smem_desc(smem_u32(sA), chunk_bytes, 1024, kSwizzle128B);
             const uint64_t b_desc0 = make_smem_desc(smem_u32(sB), G::LBO_B, 128, kSwizzleNone);
             const uint32_t a_stage_step = (uint32_t)stage_bytes >> 4;
-            uint32_t it = 0;
-            int s = 0, a = 0;
-            uint32_t ph = 0, aph = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+            const int me = warp - kMmaWarp;
+            // total rows this CTA streams
+            uint32_t total = 0;
+            for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x) {
                 int f, y0, x0, rows;
                 decode_tile(p, t, f, y0, x0, rows);
-                for (int r = 0; r < rows; ++r, ++it) {
+                total += rows;
+            }
+            int s = me % p.stages, a = me % G::ACC_SLOTS;
+            uint32_t ph = (me / p.stages) & 1, aph = (me / G::ACC_SLOTS) & 1;
+            bool ok = true;
+            for (uint32_t it = me; it < total && ok; it += kNumMmaWarps) {
 #ifdef SR_PROFILE_ROLES
-                    if (debug_mode >= 1) {
-                        if (!(ok = mbar_wait(&ctl.full[s], ph, abort_flag))) break;
-                        mbar_arrive(&ctl.empty[s]);
-                        if (++s == p.stages) { s = 0; ph ^= 1; }
-                        continue;
-                    }
-#endif
-                    if (!(ok = PROF_WAIT(mbar_wait(&ctl.acc_empty[a], aph ^ 1, abort_flag)))) break;
-                    if (!(ok = PROF_WAIT(mbar_wait(&ctl.full[s], ph, abort_flag)))) break;
-                    fence_proxy_async_smem();        // the stage was written by cp.async (generic proxy), the MMA reads it through the async proxy
-                    tc_fence_after_sync();
-                    const uint32_t taddr = tmem_base + (uint32_t)(a * G::NB);
-                    uint64_t ad = a_desc0 + (uint64_t)((uint32_t)s * a_stage_step);
-                    uint64_t bd = b_desc0;
-                    PROF_T(tm0)
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        mma_f16_ss(taddr, ad, bd, idesc, ks > 0);
-                        ad += 2048 >> 4;
-                        bd += G::KSTEP_B >> 4;
-                    }
-                    PROF_ADD(prof_mma, tm0)
-                    PROF_T(tc0)
-                    mma_commit(&ctl.empty[s]);       // the stage may be refilled once these MMAs have read it
-                    mma_commit(&ctl.acc_full[a]);    // and the accumulator is complete
-                    PROF_ADD(prof_commit, tc0)
-                    if (++s == p.stages) { s = 0; ph ^= 1; }
-                    if (++a == G::ACC_SLOTS) { a = 0; aph ^= 1; }
+                if ((debug_mode & 15) == 1 || (debug_mode & 15) == 2) {
+                    if (!(ok = mbar_wait(&ctl.full[s], ph, abort_flag))) break;
+                    mbar_arrive(&ctl.empty[s]);
+                    s += kNumMmaWarps; if (s >= p.stages) { s -= p.stages; ph ^= 1; }
+                    continue;
                 }
+#endif
+                if (!(ok = PROF_WAIT(mbar_wait(&ctl.acc_empty[a], aph ^ 1, abort_flag)))) break;
+                if (!(ok = PROF_WAIT(mbar_wait(&ctl.full[s], ph, abort_flag)))) break;
+                fence_proxy_async_smem();        // the stage was written by cp.async (generic proxy), the MMA reads it through the async proxy
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + (uint32_t)(a * G::NB);
+                uint64_t ad = a_desc0 + (uint64_t)((uint32_t)s * a_stage_step);
+                uint64_t bd = b_desc0;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    mma_f16_ss(taddr, ad, bd, idesc, ks > 0);
+                    ad += 2048 >> 4;
+                    bd += G::KSTEP_B >> 4;
+                }
+                mma_commit(&ctl.empty[s]);       // the stage may be refilled once these MMAs have read it
+                mma_commit(&ctl.acc_full[a]);    // and the accumulator is complete
+                s += kNumMmaWarps; if (s >= p.stages) { s -= p.stages; ph ^= 1; }
+                a += kNumMmaWarps; if (a >= G::ACC_SLOTS) { a -= G::ACC_SLOTS; aph ^= 1; }
             }
             PROF_STORE(warp)
         }
         __syncwarp();
-    } else if (warp < kFirstEpiWarp) {
+      } else {
         // ===== U producers: separable bicubic of the tile + halo (clamped HR coordinates), fp32.
         // The LR window of the NEXT tile is fetched with cp.async while this tile is computed. Work is
         // flattened to one output value per loop trip so that every thread of the group stays busy.
@@ -520,13 +603,13 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
             cp_async_commit();
         };
         uint32_t ti = 0;
-        if ((int)blockIdx.x < p.num_tiles) prefetch_lr(blockIdx.x, 0);
-        for (int t = blockIdx.x; t < p.num_tiles; t += gridDim.x, ++ti) {
+        if ((int)blockIdx.x < my_tiles) prefetch_lr(blockIdx.x, 0);
+        for (int t = blockIdx.x; t < my_tiles; t += gridDim.x, ++ti) {
             LrWindow g;
             lr_window<K>(p, t, g);
             const int ub = ti & 1;
             const uint32_t uph = (ti >> 1) & 1;
-            const bool has_next = t + (int)gridDim.x < p.num_tiles;
+            const bool has_next = t + (int)gridDim.x < my_tiles;
             // every thread is past the previous tile's passes before its LR buffer, scratch and tables are reused
             bool ok = PROF_WAIT(mbar_wait(&ctl.u_empty[ub], uph ^ 1, abort_flag));
             ok = named_barrier_and(1, NU, ok);
@@ -538,8 +621,7 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
                 if (i < G::UW) {
                     const int Xc = clampi(g.x0 - G::P + i, 0, pb.W - 1);
                     const int q = fast_div(Xc, pb.r, p.r_magic), px = Xc - q * pb.r;
-                    ctl.hx_off[i] = q + pb.ph.base[px] - g.col_lo;
-                    ctl.hx_w[i] = make_float4(pb.ph.w[px][0], pb.ph.w[px][1], pb.ph.w[px][2], pb.ph.w[px][3]);
+                    ctl.hx_off[i] = (q + pb.ph.base[px] - g.col_lo) | (px << 16);
                 } else {
                     const int uy = i - G::UW;
                     const int Yc = clampi(g.y0 - G::P + uy, 0, pb.H - 1);
@@ -560,27 +642,27 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
 #pragma unroll 2
             for (int o = ut; o < hrows * UW4; o += NU) {
                 const int row = o / UW4, ux = (o - row * UW4) * 4;
-                const int4 off = *reinterpret_cast<const int4*>(&ctl.hx_off[ux]);
+                const int4 op = *reinterpret_cast<const int4*>(&ctl.hx_off[ux]);   // offset | phase << 16, four columns
                 const float* Lr = Lb + row * p.tcols;
                 float4 out;
                 {
-                    const float4 w = ctl.hx_w[ux];
-                    const float* src = Lr + off.x;
+                    const float4 w = ctl.wtab[op.x >> 16];
+                    const float* src = Lr + (op.x & 0xFFFF);
                     out.x = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
                 }
                 {
-                    const float4 w = ctl.hx_w[ux + 1];
-                    const float* src = Lr + off.y;
+                    const float4 w = ctl.wtab[op.y >> 16];
+                    const float* src = Lr + (op.y & 0xFFFF);
                     out.y = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
                 }
                 {
-                    const float4 w = ctl.hx_w[ux + 2];
-                    const float* src = Lr + off.z;
+                    const float4 w = ctl.wtab[op.z >> 16];
+                    const float* src = Lr + (op.z & 0xFFFF);
                     out.z = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
                 }
                 {
-                    const float4 w = ctl.hx_w[ux + 3];
-                    const float* src = Lr + off.w;
+                    const float4 w = ctl.wtab[op.w >> 16];
+                    const float* src = Lr + (op.w & 0xFFFF);
                     out.w = fmaf(w.w, src[3], fmaf(w.z, src[2], fmaf(w.y, src[1], w.x * src[0])));
                 }
                 *reinterpret_cast<float4*>(sT + row * G::UW + ux) = out;
@@ -617,7 +699,9 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
         }
         cp_async_wait<0>();
         PROF_STORE(warp)
+      }
     } else {
+        setmaxnreg_inc<kRegsEpi>();
         // ===== epilogue: thread = one pixel column of the tile (TMEM lane); two groups of four warps own the
         // upper and the lower half of a tile and walk their rows top to bottom
         EpiCtx e;
@@ -629,11 +713,45 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
         e.tmem_lane_base = tmem_base + ((uint32_t)(e.quarter * 32) << 16);
         uint32_t it_base = 0, ti = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++ti) {
+        for (int t = blockIdx.x; t < my_tiles && ok; t += gridDim.x, ++ti) {
             int f, y0, x0, rows;
             decode_tile(p, t, f, y0, x0, rows);
             const int ub = ti & 1;
             const uint32_t uph = (ti >> 1) & 1;
+#ifdef SR_PROFILE_ROLES
+            if ((debug_mode & 15) == 3) {
+                const int h1d = rows > kHalf ? rows - kHalf : 0;
+                const int mine = e.group ? h1d : rows - h1d;
+                for (int j = 0; j < mine && ok; ++j) {
+                    const uint32_t it = it_base + item_of_half_row(j, e.group, h1d);
+                    ok = mbar_wait_warp(&ctl.acc_full[it % G::ACC_SLOTS], (it / G::ACC_SLOTS) & 1, abort_flag);
+                    if (ok) mbar_arrive(&ctl.acc_empty[it % G::ACC_SLOTS]);
+                }
+                it_base += rows;
+                continue;
+            }
+            if ((debug_mode & 15) == 4) {
+                const int h1d = rows > kHalf ? rows - kHalf : 0;
+                const int mine = e.group ? h1d : rows - h1d;
+                float sink = 0.f;
+                for (int j = 0; j < mine && ok; ++j) {
+                    const uint32_t it = it_base + item_of_half_row(j, e.group, h1d);
+                    ok = mbar_wait_warp(&ctl.acc_full[it % G::ACC_SLOTS], (it / G::ACC_SLOTS) & 1, abort_flag);
+                    if (ok) {
+                        tc_fence_after_sync();
+                        float F[G::NPAD];
+                        load_filter<K>(e.tmem_lane_base + (uint32_t)((it % G::ACC_SLOTS) * G::NB), F);
+                        tc_fence_before_sync();
+                        mbar_arrive(&ctl.acc_empty[it % G::ACC_SLOTS]);
+                        for (int q = 0; q < G::kk; ++q) sink += F[q];
+                    }
+                }
+                if (sink == 123.456f) p.out[0] = sink;
+                it_base += rows;
+                continue;
+            }
+            if ((debug_mode & 15) != 5)
+#endif
             ok = PROF_WAIT(mbar_wait_warp(&ctl.u_full[ub], uph, abort_flag));
             if (!ok) break;
             const int h1 = rows > kHalf ? rows - kHalf : 0;
@@ -643,7 +761,11 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
             const bool in_x = x0 + e.x < pb.W;
             float* dst0 = p.out + ((int64_t)f * C) * e.HW + (int64_t)(y0 + r0) * pb.W + x0 + e.x;
             if (K <= 5 && C == 3) {
+                #ifdef SR_PROFILE_ROLES
+                ok = epilogue_half_windowed<K>(ctl, e, Ub, dst0, pb.W, my_rows, h1, it_base, in_x, abort_flag, &prof_wait);
+#else
                 ok = epilogue_half_windowed<K>(ctl, e, Ub, dst0, pb.W, my_rows, h1, it_base, in_x, abort_flag);
+#endif
             } else {
                 for (int j = 0; j < my_rows; ++j) {
                     const uint32_t it = it_base + item_of_half_row(j, e.group, h1);
@@ -667,15 +789,15 @@ regress_umma_kernel(const __grid_constant__ UmmaParams p)
                 }
             }
             it_base += rows;
+#ifdef SR_PROFILE_ROLES
+            if ((debug_mode & 15) == 5) continue;
+#endif
             if (ok) mbar_arrive(&ctl.u_empty[ub]);
         }
         PROF_STORE(warp)
     }
 
     // ---------------------------------------------------------------- teardown
-#ifdef SR_PROFILE_ROLES
-teardown:
-#endif
     __syncwarp();
     tc_fence_before_sync();
     __syncthreads();
@@ -695,6 +817,23 @@ teardown:
 
 // ---- host side -------------------------------------------------------------------------------------------------------
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
+}
+
 struct DeviceInfo { int sms = 0, cc_major = 0, smem_optin = 0; bool ok = false; };
 
 const DeviceInfo& device_info()
@@ -711,6 +850,17 @@ const DeviceInfo& device_info()
         d.ok = true;
     }
     return d;
+}
+
+// Share of a stage's planes that goes through TMA (the rest through cp.async); SR_TMA_SHARE overrides (0..100).
+int tma_share_percent()
+{
+    static int v = [] {
+        const char* e = getenv("SR_TMA_SHARE");
+        int x = e ? atoi(e) : 50;
+        return x < 0 ? 0 : (x > 100 ? 100 : x);
+    }();
+    return v;
 }
 
 int trows_for(int k, int r) { return (TH + (k - 1) - 1) / r + 5; }
@@ -736,30 +886,30 @@ void contraction_shape(int mode, const Problem& pb, int& natoms, int& gather)
     }
 }
 
-template <int K> int stages_for(int c, int dpad, int r, int smem_optin)
+template <int K> int stages_for(int c, int dpad, int rows_alloc, int r, int smem_optin)
 {
     const size_t fixed = fixed_smem_bytes<K>(c, dpad, r) + kStaticReserve;
     if (fixed >= (size_t)smem_optin) return 0;
-    const int s = (int)(((size_t)smem_optin - fixed) / ((size_t)dpad * 256));
+    const int s = (int)(((size_t)smem_optin - fixed) / ((size_t)rows_alloc * 256));
     return s > kMaxStages ? kMaxStages : s;
 }
 
-int stages_for_k(int k, int c, int dpad, int r, int smem_optin)
+int stages_for_k(int k, int c, int dpad, int rows_alloc, int r, int smem_optin)
 {
     switch (k) {
-    case 1: return stages_for<1>(c, dpad, r, smem_optin);
-    case 3: return stages_for<3>(c, dpad, r, smem_optin);
-    case 5: return stages_for<5>(c, dpad, r, smem_optin);
-    case 7: return stages_for<7>(c, dpad, r, smem_optin);
+    case 1: return stages_for<1>(c, dpad, rows_alloc, r, smem_optin);
+    case 3: return stages_for<3>(c, dpad, rows_alloc, r, smem_optin);
+    case 5: return stages_for<5>(c, dpad, rows_alloc, r, smem_optin);
+    case 7: return stages_for<7>(c, dpad, rows_alloc, r, smem_optin);
     default: return 0;
     }
 }
 
 template <int K>
-cudaError_t launch_k(UmmaParams& prm, cudaStream_t st)
+cudaError_t launch_k(const CUtensorMap& map_lead, UmmaParams& prm, cudaStream_t st)
 {
     const DeviceInfo& di = device_info();
-    const size_t smem = fixed_smem_bytes<K>(prm.pb.c, prm.dpad, prm.pb.r) + (size_t)prm.stages * prm.dpad * 256;
+    const size_t smem = fixed_smem_bytes<K>(prm.pb.c, prm.dpad, prm.pb.r) + (size_t)prm.stages * prm.rows_alloc * 256;
     auto kern = regress_umma_kernel<K>;
     static bool configured[64] = {false};   // per template instance and device; the maximum is requested once
     int dev = 0;
@@ -770,7 +920,7 @@ cudaError_t launch_k(UmmaParams& prm, cudaStream_t st)
         configured[dev] = true;
     }
     const int grid = prm.num_tiles < di.sms ? prm.num_tiles : di.sms;
-    kern<<<grid, kThreads, smem, st>>>(prm);
+    kern<<<grid, kThreads, smem, st>>>(map_lead, prm);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -801,7 +951,7 @@ bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& p
     int natoms, gather;
     contraction_shape(mode, pb, natoms, gather);
     const int dpad = (natoms + 15) / 16 * 16;
-    return stages_for_k(pb.k, pb.c, dpad, pb.r, di.smem_optin) >= 2;
+    return stages_for_k(pb.k, pb.c, dpad, (natoms + 7) / 8 * 8, pb.r, di.smem_optin) >= 2;
 }
 
 cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, const uint8_t* idx, const float* gamma,
@@ -818,7 +968,8 @@ cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, con
     prm.planes = (mode == kModeGlobal && (pb.flags & SR_COEF_COMPACT)) ? pb.s : pb.D;
     prm.coef = static_cast<const __half*>(coef);
     prm.dpad = (prm.natoms + 15) / 16 * 16;
-    prm.stages = stages_for_k(pb.k, pb.c, prm.dpad, pb.r, di.smem_optin);
+    prm.rows_alloc = (prm.natoms + 7) / 8 * 8;
+    prm.stages = stages_for_k(pb.k, pb.c, prm.dpad, prm.rows_alloc, pb.r, di.smem_optin);
     prm.trows = trows_for(pb.k, pb.r);
     prm.tcols = tcols_for(pb.k, pb.r);
     prm.r_magic = pb.r > 1 ? (uint32_t)((0x100000000ull + pb.r - 1) / pb.r) : 0u;
@@ -827,11 +978,29 @@ cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, con
     prm.tiles_y = (pb.H + TH - 1) / TH;
     prm.num_tiles = prm.tiles_x * prm.tiles_y * pb.n;
 
+    // Split of the coefficient stream between the SM's two load paths: the leading planes of a stage through one
+    // TMA box per 64-pixel chunk, the rest through cp.async. Subsets gathered plane by plane use cp.async only.
+    CUtensorMap map_lead{};
+    prm.tma_rows = 0;
+    if (!prm.gather_planes && encode_fn() && prm.natoms >= 16) {
+        int lead = (prm.natoms * tma_share_percent() / 100) / 8 * 8;
+        if (lead > 0) {
+            const cuuint64_t dims[4] = {(cuuint64_t)pb.W, (cuuint64_t)pb.H, (cuuint64_t)prm.planes, (cuuint64_t)pb.n};
+            const cuuint64_t strides[3] = {(cuuint64_t)pb.W * 2, (cuuint64_t)pb.W * pb.H * 2,
+                                           (cuuint64_t)pb.W * pb.H * 2 * prm.planes};
+            const cuuint32_t es[4] = {1, 1, 1, 1};
+            const cuuint32_t box[4] = {64, 1, (cuuint32_t)lead, 1};
+            if (encode_fn()(&map_lead, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(coef), dims, strides, box, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+                prm.tma_rows = lead;
+        }
+    }
     switch (pb.k) {
-    case 1: return launch_k<1>(prm, st);
-    case 3: return launch_k<3>(prm, st);
-    case 5: return launch_k<5>(prm, st);
-    case 7: return launch_k<7>(prm, st);
+    case 1: return launch_k<1>(map_lead, prm, st);
+    case 3: return launch_k<3>(map_lead, prm, st);
+    case 5: return launch_k<5>(map_lead, prm, st);
+    case 7: return launch_k<7>(map_lead, prm, st);
     default: return cudaErrorNotSupported;
     }
 }
