@@ -1,6 +1,14 @@
 // Per-pixel top-s selection by coefficient magnitude, ties to the lower atom index, rank order out.
 // Key of atom l = (bit pattern with the sign cleared) * 256 + (255 - l): one integer whose order is
 // exactly "larger magnitude first, then lower index"; keys of one pixel are distinct.
+//
+// Fast path (binary16 coefficients, s <= 16, even W): one thread owns two neighbouring pixels (one 4-byte load per
+// plane, a full 128-byte line per warp), keeps their s best keys sorted in registers and merges every group of S
+// planes with branch-free sorting networks of integer max / min:
+//   sort the S new keys (19 compare-exchanges for S = 8), max against the reversed running list (S ops, gives a
+//   bitonic sequence holding the S best of both), bitonic-merge it back to sorted order (S/2 * log2 S exchanges).
+// Per pixel and plane that is about 8.75 min/max for S = 8 (630 per pixel at D = 72) against 16 for plain insertion.
+// The kernel is bound by the integer ALU rate or by HBM, whichever is slower for the shape.
 #include "sr_common.cuh"
 
 namespace sr {
@@ -18,7 +26,110 @@ __device__ __forceinline__ typename KeyOf<CoefT>::type make_key(CoefT v, int l)
     return (KeyT)(((KeyT)mag_bits(v) << 8) | (KeyT)(255 - l));
 }
 
-// s <= SMAX: sorted list in registers, one branch-free insertion per atom.
+// ---- sorting networks on int keys (descending) -----------------------------------------------------------------------
+
+__device__ __forceinline__ void cx(int& a, int& b)    // afterwards a >= b
+{
+    const int hi = max(a, b), lo = min(a, b);
+    a = hi;
+    b = lo;
+}
+
+template <int S> __device__ __forceinline__ void sort_desc(int* k);
+
+template <> __device__ __forceinline__ void sort_desc<4>(int* k)
+{
+    cx(k[0], k[1]); cx(k[2], k[3]);
+    cx(k[0], k[2]); cx(k[1], k[3]);
+    cx(k[1], k[2]);
+}
+
+template <> __device__ __forceinline__ void sort_desc<8>(int* k)   // 19 exchanges
+{
+    cx(k[0], k[1]); cx(k[2], k[3]); cx(k[4], k[5]); cx(k[6], k[7]);
+    cx(k[0], k[2]); cx(k[1], k[3]); cx(k[4], k[6]); cx(k[5], k[7]);
+    cx(k[1], k[2]); cx(k[5], k[6]);
+    cx(k[0], k[4]); cx(k[1], k[5]); cx(k[2], k[6]); cx(k[3], k[7]);
+    cx(k[2], k[4]); cx(k[3], k[5]);
+    cx(k[1], k[2]); cx(k[3], k[4]); cx(k[5], k[6]);
+}
+
+// Sorts a bitonic sequence of S keys into descending order.
+template <int S> __device__ __forceinline__ void bitonic_merge_desc(int* k)
+{
+#pragma unroll
+    for (int d = S / 2; d >= 1; d >>= 1)
+#pragma unroll
+        for (int i = 0; i < S; ++i)
+            if ((i & d) == 0) cx(k[i], k[i + d]);
+}
+
+template <> __device__ __forceinline__ void sort_desc<16>(int* k)   // two sorted halves, then a bitonic merge
+{
+    sort_desc<8>(k);
+    sort_desc<8>(k + 8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const int t = k[8 + i]; k[8 + i] = k[15 - i]; k[15 - i] = t; }   // second half ascending
+    bitonic_merge_desc<16>(k);
+}
+
+// top[] (sorted) <- the S best of top[] and grp[] (grp sorted descending)
+template <int S> __device__ __forceinline__ void merge_top(int* top, const int* grp)
+{
+#pragma unroll
+    for (int i = 0; i < S; ++i) top[i] = max(top[i], grp[S - 1 - i]);
+    bitonic_merge_desc<S>(top);
+}
+
+// Two pixels per thread, binary16, s <= S, W even.
+template <int S>
+__global__ void __launch_bounds__(256)
+select_pair_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
+                   const __grid_constant__ Problem pb)
+{
+    const int64_t HW = (int64_t)pb.H * pb.W;
+    const int64_t pairs_per_frame = HW / 2;
+    const int64_t total = (int64_t)pb.n * pairs_per_frame;
+    const int D = pb.D, s = pb.s;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t f = t / pairs_per_frame, pix = (t - f * pairs_per_frame) * 2;
+        const __half* cp = coef + f * D * HW + pix;
+        int ta[S], tb[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1;
+        for (int l0 = 0; l0 < D; l0 += S) {
+            uint32_t w[S];
+#pragma unroll
+            for (int i = 0; i < S; ++i)
+                w[i] = (l0 + i < D) ? __ldg(reinterpret_cast<const uint32_t*>(cp + (int64_t)(l0 + i) * HW)) : 0u;
+            int ga[S], gb[S];
+#pragma unroll
+            for (int i = 0; i < S; ++i) {
+                const int tag = 255 - (l0 + i);
+                ga[i] = (l0 + i < D) ? (int)(((w[i] << 8) & 0x7FFF00u) | (uint32_t)tag) : -1;
+                gb[i] = (l0 + i < D) ? (int)(((w[i] >> 8) & 0x7FFF00u) | (uint32_t)tag) : -1;
+            }
+            sort_desc<S>(ga);
+            sort_desc<S>(gb);
+            merge_top<S>(ta, ga);
+            merge_top<S>(tb, gb);
+        }
+#pragma unroll
+        for (int q = 0; q < S; ++q) {
+            if (q < s) {
+                const int a = 255 - (ta[q] & 255), b = 255 - (tb[q] & 255);
+                const int64_t o = (f * s + q) * HW + pix;
+                *reinterpret_cast<uchar2*>(idx + o) = make_uchar2((unsigned char)a, (unsigned char)b);
+                if (sel) {
+                    const __half va = __ldg(cp + (int64_t)a * HW), vb = __ldg(cp + (int64_t)b * HW + 1);
+                    *reinterpret_cast<__half2*>(sel + o) = __halves2half2(va, vb);
+                }
+            }
+        }
+    }
+}
+
+// s <= SMAX: sorted list in registers, one branch-free insertion per atom (any dtype, any W).
 template <typename CoefT, int SMAX>
 __global__ void __launch_bounds__(256)
 select_insert_kernel(const CoefT* __restrict__ coef, uint8_t* __restrict__ idx, CoefT* __restrict__ sel,
@@ -82,12 +193,22 @@ select_scan_kernel(const CoefT* __restrict__ coef, uint8_t* __restrict__ idx, Co
     }
 }
 
+int sm_count()
+{
+    static int sms[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms[dev] = 148;
+    return sms[dev];
+}
+
 template <typename CoefT>
 cudaError_t launch_sel(const void* coef, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
 {
     const int64_t total = (int64_t)pb.n * pb.H * pb.W;
     int64_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 64) blocks = 148 * 64;
+    const int64_t cap = (int64_t)sm_count() * 64;
+    if (blocks > cap) blocks = cap;
     const CoefT* c = (const CoefT*)coef;
     CoefT* sl = (CoefT*)sel;
     if (pb.s <= 4) select_insert_kernel<CoefT, 4><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
@@ -98,11 +219,36 @@ cudaError_t launch_sel(const void* coef, uint8_t* idx, void* sel, const Problem&
     return cudaGetLastError();
 }
 
+// binary16 fast path: needs 4-byte aligned pixel pairs in every plane and in the outputs
+bool pair_path_ok(const void* coef, const uint8_t* idx, const void* sel, const Problem& pb)
+{
+    return pb.s <= 16 && (pb.W & 1) == 0 && (reinterpret_cast<uintptr_t>(coef) & 3) == 0 &&
+           (reinterpret_cast<uintptr_t>(idx) & 1) == 0 && (reinterpret_cast<uintptr_t>(sel) & 3) == 0;
+}
+
+cudaError_t launch_pair(const void* coef, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
+{
+    const int64_t total = (int64_t)pb.n * pb.H * pb.W / 2;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    const __half* c = (const __half*)coef;
+    __half* sl = (__half*)sel;
+    if (pb.s <= 4) select_pair_kernel<4><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
+    else if (pb.s <= 8) select_pair_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
+    else select_pair_kernel<16><<<(unsigned)blocks, 256, 0, st>>>(c, idx, sl, pb);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 } // namespace
 
 cudaError_t launch_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
 {
-    if (coef_dtype == SR_F16) return launch_sel<__half>(coef, idx, sel, pb, st);
+    if (coef_dtype == SR_F16) {
+        if (pair_path_ok(coef, idx, sel, pb)) return launch_pair(coef, idx, sel, pb, st);
+        return launch_sel<__half>(coef, idx, sel, pb, st);
+    }
     return launch_sel<float>(coef, idx, sel, pb, st);
 }
 
