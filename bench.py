@@ -65,14 +65,19 @@ NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": None, "select": None, "compact": None, "
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs.
+
+    The sampler starts before the warm-up; `stop(t0, t1)` keeps the samples whose timestamps fall inside the timed
+    region [t0, t1] (host wall-clock seconds) and falls back to the busiest half when the region was shorter than
+    the sampling period.
+    """
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_uuid: str | None):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"]
         if gpu_uuid:
             cmd += ["-i", gpu_uuid]
         try:
@@ -80,9 +85,17 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self) -> dict:
+    def wait_first_sample(self, timeout_s: float = 5.0):
+        t0 = time.time()
+        while self.proc is not None and time.time() - t0 < timeout_s:
+            if os.path.getsize(self.tmp.name) > 0:
+                return
+            time.sleep(0.02)
+
+    def stop(self, t0: float, t1: float) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -90,27 +103,31 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, smax, reasons, power = [], [], set(), []
+        import datetime
+        rows = []
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.tmp.read().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                smax.append(float(parts[1]))
-                power.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]),
+                             [n for n, v in zip(names, parts[4:8]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.tmp.close()
         os.unlink(self.tmp.name)
-        # the busiest half of the samples: the sampler also sees the idle time around the timed region
-        busy = sorted(sm)[len(sm) // 2:] if sm else []
-        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(smax) if smax else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        how = "samples inside the timed region"
+        if not inside and rows:
+            how = "timed region shorter than the sampling period: busiest half of all samples"
+            inside = sorted(rows, key=lambda r: r[1])[len(rows) // 2:]
+        reasons = sorted({n for r in inside for n in r[4]})
+        return {"sm_mhz": statistics.median([r[1] for r in inside]) if inside else None,
+                "sm_max_mhz": max([r[2] for r in rows]) if rows else None,
+                "power_w_max": max([r[3] for r in inside]) if inside else None,
+                "samples": len(inside), "reasons": reasons, "how": how}
 
 
 def oracle_step(oracle, wl, lr, dict_, coef, S, gamma, rows: int | None, threads: int = 0):
@@ -192,8 +209,8 @@ def workload_config(wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--paths", default=",".join(PATHS), help="comma-separated subset of the step's paths (profiling)")
@@ -275,28 +292,32 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        step(sets[i % nsets])
-    barrier()
-
     uuid = None
     try:
         uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
     except Exception:
         pass
     sampler = ClockSampler(uuid) if rank == 0 else None
+    if sampler:
+        sampler.wait_first_sample()
+    for i in range(args.warmup):
+        step(sets[i % nsets])
+    barrier()
+
     launches0 = sr.sr_launch_count()
     events = []
     barrier()
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     t_start.record()
     for i in range(args.steps):
         step(sets[i % nsets], events)
     t_end.record()
     barrier()
+    wall1 = time.time()
     elapsed_ms = t_start.elapsed_time(t_end)
     launches = sr.sr_launch_count() - launches0
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(wall0, wall1) if sampler else None
     if sr.sr_device_status() != 0:
         raise SystemExit("device status word reports an expired wait")
     if dist is not None:
