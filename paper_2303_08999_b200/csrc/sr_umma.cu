@@ -37,13 +37,27 @@ namespace {
 using namespace ptx;
 
 constexpr int TW = 128, TH = 16;
-constexpr int kThreads = 640;
 constexpr int kNumLoadWarps = 4, kMmaWarp = 4, kNumMmaWarps = 2;
-constexpr int kFirstUWarp = 6, kNumUWarps = 6, kFirstEpiWarp = 12, kNumEpiWarps = 8;
-// Registers per thread after the warpgroups re-balance the register file (setmaxnreg): 20 warps start at 96;
-// loaders and the MMA / U warpgroups give registers back, the two epilogue warpgroups take them.
-// 4*40 + 8*72 + 8*144 = 1888 <= 2048 warp-registers.
-constexpr int kRegsLoad = 40, kRegsMmaU = 72, kRegsEpi = 144;
+constexpr int kFirstUWarp = 6, kNumUWarps = 6, kFirstSelWarp = 12, kNumSelWarps = 4, kNumEpiWarps = 8;
+
+// Role layout. The selective variant (per-pixel top-s chosen inside the kernel) inserts one warpgroup of
+// "select" warps between the loaders and the MMA issuers: they rewrite each landed stage in place, zeroing the
+// coefficients that are not among the pixel's s largest, and the rest of the pipeline is the dense one.
+template <bool SEL> struct Cfg {
+    static constexpr int kFirstEpiWarp = SEL ? kFirstSelWarp + kNumSelWarps : kFirstSelWarp;   // 16 or 12
+    static constexpr int kThreads = (kFirstEpiWarp + kNumEpiWarps) * 32;                        // 768 or 640
+    // Registers per thread after setmaxnreg. setmaxnreg only moves registers inside the pool the CTA was given at
+    // launch (warps x registers-per-thread the kernel was compiled for), so the re-balanced total must not exceed
+    // it: an increase that can never be satisfied would block forever.
+    static constexpr int kRegsLaunch = SEL ? 80 : 96;       // 65536 / threads, rounded down to a multiple of 8
+    static constexpr int kRegsLoad = 40, kRegsMmaU = SEL ? 56 : 72, kRegsSel = 64, kRegsEpi = SEL ? 128 : 144;
+    static constexpr int kNumWarps = kFirstEpiWarp + kNumEpiWarps;
+    static constexpr int kPoolAfter = kNumLoadWarps * kRegsLoad + (kFirstSelWarp - kNumLoadWarps) * kRegsMmaU +
+                                      (SEL ? kNumSelWarps * kRegsSel : 0) + kNumEpiWarps * kRegsEpi;
+    static_assert(kRegsLaunch * kThreads <= 65536, "launch register count does not fit the register file");
+    static_assert(kPoolAfter <= kNumWarps * kRegsLaunch, "re-balanced registers exceed the CTA's pool");
+};
+
 constexpr int kMaxStages = 10;
 constexpr int kMaxAccSlots = 8;
 constexpr int kMaxChannels = 4;
@@ -64,6 +78,7 @@ struct UmmaParams {
                           // below dpad the last K-step's upper 8 rows read whatever follows the chunk; the matching
                           // dictionary rows are zero, so any finite bytes there contribute nothing.
     int planes;           // planes per frame in the coefficient tensor (D, or s when it is compact)
+    int sel_s;            // selective variant: atoms kept per pixel
     int tma_rows;         // leading planes of every stage that a TMA box brings in (multiple of 8; 0 = none); the
                           // rest arrive through cp.async, so that both load paths of the SM work side by side
     int gather_planes;    // 1: plane q of the contraction is plane atoms[q] of the tensor (subset of a full tensor)
@@ -78,6 +93,7 @@ struct UmmaParams {
 
 struct __align__(16) Ctl {
     uint64_t full[kMaxStages], empty[kMaxStages];
+    uint64_t ready[kMaxStages];   // selective variant: the stage has been masked and may be multiplied
     uint64_t acc_full[kMaxAccSlots], acc_empty[kMaxAccSlots];
     uint64_t u_full[2], u_empty[2];
     uint32_t tmem_base;
@@ -255,6 +271,103 @@ __device__ __forceinline__ void patch_dot(const float* F, const float* u, int ch
     }
 }
 
+// ---- per-pixel top-s masking of a staged row (selective variant) -----------------------------------------------------
+
+__device__ __forceinline__ void cx_h2(__half2& a, __half2& b)    // afterwards a >= b in both halves
+{
+    const __half2 hi = __hmax2(a, b), lo = __hmin2(a, b);
+    a = hi;
+    b = lo;
+}
+
+__device__ __forceinline__ void sort8_desc_h2(__half2 (&k)[8])   // 19 exchanges
+{
+    cx_h2(k[0], k[1]); cx_h2(k[2], k[3]); cx_h2(k[4], k[5]); cx_h2(k[6], k[7]);
+    cx_h2(k[0], k[2]); cx_h2(k[1], k[3]); cx_h2(k[4], k[6]); cx_h2(k[5], k[7]);
+    cx_h2(k[1], k[2]); cx_h2(k[5], k[6]);
+    cx_h2(k[0], k[4]); cx_h2(k[1], k[5]); cx_h2(k[2], k[6]); cx_h2(k[3], k[7]);
+    cx_h2(k[2], k[4]); cx_h2(k[3], k[5]);
+    cx_h2(k[1], k[2]); cx_h2(k[3], k[4]); cx_h2(k[5], k[6]);
+}
+
+__device__ __forceinline__ void bitonic_merge8_desc_h2(__half2 (&k)[8])
+{
+#pragma unroll
+    for (int d = 4; d >= 1; d >>= 1)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if ((i & d) == 0) cx_h2(k[i], k[i + d]);
+}
+
+__device__ __forceinline__ __half2 h2_from_bits(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+__device__ __forceinline__ uint32_t bits_from_h2(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
+// Masks two independent pixel pairs (columns `colA`, `colB`: pointers at (atom 0, two neighbouring pixels) of a
+// stage; atom l of a pair sits at col + l*128 + ((c16 ^ (l & 7)) << 4)) so that two sorting networks are in flight
+// per thread. Keeps, per pixel, the s (<= 8) coefficients of largest magnitude (ties: lower atom index first) and
+// zeroes the rest. Magnitudes are compared as positive binary16 numbers, which orders finite values exactly like
+// their bit patterns.
+__device__ __forceinline__ void select_mask_stage(uint8_t* colA, uint32_t c16A, uint8_t* colB, uint32_t c16B, int natoms, int s)
+{
+    auto wordA = [&](int l) -> uint32_t* {
+        return reinterpret_cast<uint32_t*>(colA + (uint32_t)l * 128u + (((c16A ^ (uint32_t)(l & 7))) << 4));
+    };
+    auto wordB = [&](int l) -> uint32_t* {
+        return reinterpret_cast<uint32_t*>(colB + (uint32_t)l * 128u + (((c16B ^ (uint32_t)(l & 7))) << 4));
+    };
+    const __half2 zero = h2_from_bits(0u);
+    // The running list starts with 8 - s entries of +infinity: they stay on top, so the s-th largest real
+    // magnitude always ends up in slot 7 and no slot has to be picked at run time.
+    const __half2 inf = h2_from_bits(0x7C007C00u);
+    __half2 topA[8], topB[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) topA[i] = topB[i] = (i < 8 - s) ? inf : zero;
+    for (int l0 = 0; l0 < natoms; l0 += 8) {
+        __half2 gA[8], gB[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            gA[i] = (l0 + i < natoms) ? h2_from_bits(*wordA(l0 + i) & 0x7FFF7FFFu) : zero;
+            gB[i] = (l0 + i < natoms) ? h2_from_bits(*wordB(l0 + i) & 0x7FFF7FFFu) : zero;
+        }
+        sort8_desc_h2(gA);
+        sort8_desc_h2(gB);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            topA[i] = __hmax2(topA[i], gA[7 - i]);
+            topB[i] = __hmax2(topB[i], gB[7 - i]);
+        }
+        bitonic_merge8_desc_h2(topA);
+        bitonic_merge8_desc_h2(topB);
+    }
+    // tau = s-th largest magnitude; need = how many coefficients equal to tau are kept = s - #(magnitudes > tau)
+    // = 8 - #(list entries > tau), the virtual infinities included
+    const __half2 tauA = topA[7], tauB = topB[7];
+    __half2 gtA = zero, gtB = zero;
+#pragma unroll
+    for (int i = 0; i < 7; ++i) { gtA = __hadd2(gtA, __hgt2(topA[i], tauA)); gtB = __hadd2(gtB, __hgt2(topB[i], tauB)); }
+    const __half2 eight = __float2half2_rn(8.f);
+    const __half2 needA = __hsub2(eight, gtA), needB = __hsub2(eight, gtB);
+    // above tau everything passes; once `need` ties have passed, the threshold moves one ulp up for that pixel
+    const uint32_t tA = bits_from_h2(tauA), tB = bits_from_h2(tauB);
+    const uint32_t tA1 = tA + 0x00010001u, tB1 = tB + 0x00010001u;     // next representable magnitude (per half)
+    uint32_t thrA = tA, thrB = tB;                                     // need >= 1: tau itself is one of the ties
+    __half2 cntA = zero, cntB = zero;
+#pragma unroll 4
+    for (int l = 0; l < natoms; ++l) {
+        uint32_t* wa = wordA(l);
+        uint32_t* wb = wordB(l);
+        const uint32_t a = *wa, b = *wb;
+        const __half2 ma = h2_from_bits(a & 0x7FFF7FFFu), mb = h2_from_bits(b & 0x7FFF7FFFu);
+        *wa = a & __hge2_mask(ma, h2_from_bits(thrA));
+        *wb = b & __hge2_mask(mb, h2_from_bits(thrB));
+        cntA = __hadd2(cntA, __heq2(ma, tauA));
+        cntB = __hadd2(cntB, __heq2(mb, tauB));
+        const uint32_t exA = __hge2_mask(cntA, needA), exB = __hge2_mask(cntB, needB);
+        thrA = (tA & ~exA) | (tA1 & exA);
+        thrB = (tB & ~exB) | (tB1 & exB);
+    }
+}
+
 struct EpiCtx {
     int quarter, group, x;
     int64_t HW;
@@ -383,11 +496,13 @@ __device__ int g_debug_mode = 0;   // 1: TMA streaming only (no MMA, no U, no ep
 #define PROF_STORE2(role, a, b)
 #endif
 
-template <int K>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int K, bool SEL>
+__global__ void __launch_bounds__(Cfg<SEL>::kThreads, 1)
 regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_constant__ UmmaParams p)
 {
     using G = Geo<K>;
+    using CF = Cfg<SEL>;
+    constexpr int kThreads = CF::kThreads, kFirstEpiWarp = CF::kFirstEpiWarp;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ Ctl ctl;
 
@@ -410,7 +525,7 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_c
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
-        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], kNumLoadWarps * 32 + (p.tma_rows > 0 ? 1 : 0)); mbar_init(&ctl.empty[i], 1); }
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.full[i], kNumLoadWarps * 32 + (p.tma_rows > 0 ? 1 : 0)); mbar_init(&ctl.empty[i], 1); mbar_init(&ctl.ready[i], 32); }
         for (int i = 0; i < kMaxAccSlots; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], 128); }
         for (int i = 0; i < 2; ++i) { mbar_init(&ctl.u_full[i], kNumUWarps * 32); mbar_init(&ctl.u_empty[i], kNumEpiWarps * 32); }
         ctl.abort_flag = 0;
@@ -472,7 +587,7 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_c
     // Each role's branch starts by re-balancing the register file for its warpgroup (all four warps of a
     // warpgroup execute the same setmaxnreg instruction).
     if (warp < kNumLoadWarps) {
-        setmaxnreg_dec<kRegsLoad>();
+        setmaxnreg_dec<CF::kRegsLoad>();
         // ===== coefficient producers: 128 threads, thread = (16-byte column c16 of the 128-pixel row, atom l0 + 8k)
         // A stage is [chunk of 64 pixels][atom][128 B]; within a 1024-byte group of 8 atoms the 16-byte columns are
         // XOR-swizzled with the atom index (the 128-byte swizzle the MMA descriptor names).
@@ -526,8 +641,8 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_c
         }
         cp_async_wait_all();                                 // nothing of this thread is in flight at exit
         PROF_STORE(warp)
-    } else if (warp < kFirstEpiWarp) {
-      setmaxnreg_dec<kRegsMmaU>();
+    } else if (warp < kFirstSelWarp) {
+      setmaxnreg_dec<CF::kRegsMmaU>();
       if (warp < kMmaWarp + kNumMmaWarps) {
         // ===== MMA issuers: warp kMmaWarp + m takes the rows whose running index is m modulo kNumMmaWarps
         if (lane == 0) {
@@ -559,7 +674,7 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_c
                 }
 #endif
                 if (!(ok = PROF_WAIT(mbar_wait(&ctl.acc_empty[a], aph ^ 1, abort_flag)))) break;
-                if (!(ok = PROF_WAIT(mbar_wait(&ctl.full[s], ph, abort_flag)))) break;
+                if (!(ok = PROF_WAIT(mbar_wait(SEL ? &ctl.ready[s] : &ctl.full[s], ph, abort_flag)))) break;
                 fence_proxy_async_smem();        // the stage was written by cp.async (generic proxy), the MMA reads it through the async proxy
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (uint32_t)(a * G::NB);
@@ -700,8 +815,39 @@ regress_umma_kernel(const __grid_constant__ CUtensorMap map_lead, const __grid_c
         cp_async_wait<0>();
         PROF_STORE(warp)
       }
+    } else if (SEL && warp < kFirstEpiWarp) {
+        setmaxnreg_dec<CF::kRegsSel>();
+        // ===== select warps: one warp per stage (32 threads x 2 pixel pairs); warp w takes the stages whose
+        // running index is w modulo 4. Per pixel: the s-th largest magnitude tau by sorting networks on packed
+        // binary16 magnitudes, then every coefficient below tau, and every tie with tau beyond the first `need` in
+        // atom order, is zeroed in place.
+        const int me = warp - kFirstSelWarp;
+        // this thread's pixel pairs: pixels 2*lane, 2*lane+1 of the first and of the second 64-pixel chunk
+        const int px = 2 * lane;
+        const uint32_t colA = (uint32_t)((px & 7) * 2), colB = (uint32_t)(chunk_bytes + (px & 7) * 2);
+        const uint32_t c16 = (uint32_t)(px >> 3);
+        uint32_t total = 0;
+        for (int t = blockIdx.x; t < my_tiles; t += gridDim.x) {
+            int f, y0, x0, rows;
+            decode_tile(p, t, f, y0, x0, rows);
+            total += rows;
+        }
+        int s = me % p.stages;
+        uint32_t ph = (me / p.stages) & 1;
+        bool ok = true;
+        for (uint32_t it = me; it < total && ok; it += kNumSelWarps) {
+            ok = mbar_wait_warp(&ctl.full[s], ph, abort_flag);
+            if (!ok) break;
+            uint8_t* stage = sA + (size_t)s * stage_bytes;
+            select_mask_stage(stage + colA, c16, stage + colB, c16, p.natoms, p.sel_s);
+            fence_proxy_async_smem();                                    // masked stage -> tensor core (async proxy)
+            mbar_arrive(&ctl.ready[s]);
+            s += kNumSelWarps;
+            while (s >= p.stages) { s -= p.stages; ph ^= 1; }
+        }
+        PROF_STORE(warp)
     } else {
-        setmaxnreg_inc<kRegsEpi>();
+        setmaxnreg_inc<CF::kRegsEpi>();
         // ===== epilogue: thread = one pixel column of the tile (TMEM lane); two groups of four warps own the
         // upper and the lower half of a tile and walk their rows top to bottom
         EpiCtx e;
@@ -894,6 +1040,16 @@ template <int K> int stages_for(int c, int dpad, int rows_alloc, int r, int smem
     return s > kMaxStages ? kMaxStages : s;
 }
 
+// A role that takes every n-th row (two MMA issuers, four select warps) must meet every use of the stages it
+// waits on, one after the other: mbarrier waits only know the parity of a phase, so a waiter that skipped a use
+// could mistake the phase before last for the one it wants. With the stage count a multiple of n each such warp
+// owns a fixed subset of the stages.
+int usable_stages(int mode, int stages)
+{
+    const int n = (mode == kModeFusedSelect) ? kNumSelWarps : kNumMmaWarps;
+    return stages / n * n;
+}
+
 int stages_for_k(int k, int c, int dpad, int rows_alloc, int r, int smem_optin)
 {
     switch (k) {
@@ -905,12 +1061,12 @@ int stages_for_k(int k, int c, int dpad, int rows_alloc, int r, int smem_optin)
     }
 }
 
-template <int K>
-cudaError_t launch_k(const CUtensorMap& map_lead, UmmaParams& prm, cudaStream_t st)
+template <int K, bool SEL>
+cudaError_t launch_ks(const CUtensorMap& map_lead, UmmaParams& prm, cudaStream_t st)
 {
     const DeviceInfo& di = device_info();
     const size_t smem = fixed_smem_bytes<K>(prm.pb.c, prm.dpad, prm.pb.r) + (size_t)prm.stages * prm.rows_alloc * 256;
-    auto kern = regress_umma_kernel<K>;
+    auto kern = regress_umma_kernel<K, SEL>;
     static bool configured[64] = {false};   // per template instance and device; the maximum is requested once
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -920,9 +1076,15 @@ cudaError_t launch_k(const CUtensorMap& map_lead, UmmaParams& prm, cudaStream_t 
         configured[dev] = true;
     }
     const int grid = prm.num_tiles < di.sms ? prm.num_tiles : di.sms;
-    kern<<<grid, kThreads, smem, st>>>(map_lead, prm);
+    kern<<<grid, Cfg<SEL>::kThreads, smem, st>>>(map_lead, prm);
     count_launches(1);
     return cudaGetLastError();
+}
+
+template <int K>
+cudaError_t launch_k(const CUtensorMap& map_lead, UmmaParams& prm, cudaStream_t st)
+{
+    return prm.mode == kModeFusedSelect ? launch_ks<K, true>(map_lead, prm, st) : launch_ks<K, false>(map_lead, prm, st);
 }
 
 } // namespace
@@ -941,7 +1103,7 @@ extern "C" int sr_debug_role_profile(long long* device_buffer)
 
 bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& pb)
 {
-    if (mode != kModeDense && mode != kModeGlobal) return false;
+    if (mode != kModeDense && mode != kModeGlobal && !(mode == kModeFusedSelect && pb.s <= 8)) return false;
     if (coef_dtype != SR_F16) return false;
     if (pb.k > 7 || pb.c > kMaxChannels) return false;
     if ((reinterpret_cast<uintptr_t>(coef) & 15) != 0 || (pb.W & 7) != 0) return false;   // 16-byte copies: aligned base and row pitch
@@ -951,7 +1113,7 @@ bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& p
     int natoms, gather;
     contraction_shape(mode, pb, natoms, gather);
     const int dpad = (natoms + 15) / 16 * 16;
-    return stages_for_k(pb.k, pb.c, dpad, (natoms + 7) / 8 * 8, pb.r, di.smem_optin) >= 2;
+    return usable_stages(mode, stages_for_k(pb.k, pb.c, dpad, (natoms + 7) / 8 * 8, pb.r, di.smem_optin)) >= 2;
 }
 
 cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, const uint8_t* idx, const float* gamma,
@@ -964,12 +1126,13 @@ cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, con
     if (!prm.status) return cudaErrorUnknown;
     prm.pb = pb;
     prm.mode = mode;
+    prm.sel_s = pb.s;
     contraction_shape(mode, pb, prm.natoms, prm.gather_planes);
     prm.planes = (mode == kModeGlobal && (pb.flags & SR_COEF_COMPACT)) ? pb.s : pb.D;
     prm.coef = static_cast<const __half*>(coef);
     prm.dpad = (prm.natoms + 15) / 16 * 16;
     prm.rows_alloc = (prm.natoms + 7) / 8 * 8;
-    prm.stages = stages_for_k(pb.k, pb.c, prm.dpad, prm.rows_alloc, pb.r, di.smem_optin);
+    prm.stages = usable_stages(mode, stages_for_k(pb.k, pb.c, prm.dpad, prm.rows_alloc, pb.r, di.smem_optin));
     prm.trows = trows_for(pb.k, pb.r);
     prm.tcols = tcols_for(pb.k, pb.r);
     prm.r_magic = pb.r > 1 ? (uint32_t)((0x100000000ull + pb.r - 1) / pb.r) : 0u;
