@@ -26,7 +26,8 @@ def _newest(paths):
 
 def build(force: bool = False, verbose: bool = False) -> str:
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
-    hdrs = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(_ROOT, "include", "*.h"))
+    hdrs = (glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.inc")) +
+            glob.glob(os.path.join(_ROOT, "include", "*.h")))
     os.makedirs(_OBJ, exist_ok=True)
     hdr_time = _newest(hdrs) if hdrs else 0.0
     jobs = []
