@@ -50,6 +50,26 @@ def algorithmic_bytes_per_pixel(wl, path: str) -> float:
     }[path]
 
 
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank owns its own frames: the generator seed is offset by the rank (weak scaling, no data exchange)."""
+    return base_seed + rank
+
+
+def max_over_ranks(value_ms: float, dist=None, device=None) -> float:
+    """Device time of the slowest rank (the only collective on the timing path); identity without a process group."""
+    if dist is None or not dist.is_initialized():
+        return float(value_ms)
+    import torch
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, pixels_per_rank_step: int, steps: int, max_ms: float) -> float:
+    """HR megapixels per second of the whole job: all ranks' pixels over the slowest rank's time."""
+    return world * pixels_per_rank_step * steps / (max_ms * 1e-3) / 1e6
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -61,7 +81,7 @@ def load_peaks():
 
 # DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
 # kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": None, "select": None, "compact": None, "fused": None, "global": None}
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": 155.05, "select": 174.6, "compact": None, "fused": 154.8, "global": 17.1}
 
 
 class ClockSampler:
@@ -245,7 +265,7 @@ def main():
     sr.load_library()
 
     # ---- inputs: every rank owns its own frames (seed offset by rank); three rotating buffer sets
-    seed = sr_inputs.BASE_SEED + rank
+    seed = rank_seed(sr_inputs.BASE_SEED, rank)
     lr, dict_, coef = sr_inputs.make_inputs(wl, seed)
     S = np.arange(0, wl.D, max(1, wl.D // wl.s), dtype=np.uint8)[: wl.s]
     gamma = np.linspace(0.75, 1.25, wl.s).astype(np.float32)
@@ -320,10 +340,7 @@ def main():
     clocks = sampler.stop(wall0, wall1) if sampler else None
     if sr.sr_device_status() != 0:
         raise SystemExit("device status word reports an expired wait")
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, "cuda")
 
     # per-path averages from the events recorded inside the timed region
     per_path_ms = {}
@@ -355,11 +372,8 @@ def main():
         b.record()
         barrier()
         ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": world * wl.npix * e2e_steps / (ms * 1e-3) / 1e6, "unit": "MP/s",
+        ms = max_over_ranks(ms, dist, "cuda")
+        e2e = {"value": whole_job_value(world, wl.npix, e2e_steps, ms), "unit": "MP/s",
                "h2d_bytes_per_step": h_lr.numel() * 4 + h_coef.numel() * h_coef.element_size(),
                "d2h_bytes_per_step": sum(o.numel() * 4 for o in outs.values()), "steps": e2e_steps}
 
@@ -387,7 +401,7 @@ def main():
         cpu = time_oracle(wl, lr, dict_, coef, S, gamma)
 
     line = {
-        "metric": METRIC, "value": world * wl.npix * args.steps / (elapsed_ms * 1e-3) / 1e6, "unit": "MP/s",
+        "metric": METRIC, "value": whole_job_value(world, wl.npix, args.steps, elapsed_ms), "unit": "MP/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate, f16 coefficients"
         if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": dict(workload_config(wl), paths_per_step=list(active)),
