@@ -84,6 +84,29 @@ def load_peaks():
 NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": 155.05, "select": 174.6, "compact": None, "fused": 154.8, "global": 17.1}
 
 
+# Half-rate integer / binary16 max-min-compare operations per HR pixel of the two selection kernels (sorting-network
+# merges; counted in the design doc section 5) and the B200 rate of that pipe: 148 SMs x 64 lanes/clk x 1.965 GHz.
+ALU_OPS_PER_PIXEL = {"select": 630.0, "fused": 459.0}
+ALU_PEAK_GOPS = 148 * 64 * 1.965
+
+
+def path_roofline(wl, path: str, ms: float, hbm_peak: float, peak_kind: str, traffic_bytes_per_pixel):
+    """Roofline entry of one path: the slower of its bytes at HBM bandwidth and its selection ops at the ALU rate."""
+    by = algorithmic_bytes_per_pixel(wl, path) * wl.npix
+    t_hbm = by / (hbm_peak * 1e9)
+    ops = ALU_OPS_PER_PIXEL.get(path, 0.0) * wl.npix if (wl.D == 72 and wl.s == 8) else 0.0
+    t_alu = ops / (ALU_PEAK_GOPS * 1e9)
+    traffic = None if traffic_bytes_per_pixel is None else traffic_bytes_per_pixel * wl.npix
+    if t_alu > t_hbm:
+        ach = ops / (ms * 1e-3) / 1e9
+        return {"kernel": path, "bound": "alu", "achieved": ach, "peak": ALU_PEAK_GOPS, "unit": "Gop/s (max/min lanes)",
+                "frac": ach / ALU_PEAK_GOPS, "peak_kind": "derived: 148 SMs x 64 lanes/clk x 1.965 GHz", "traffic": traffic,
+                "hbm_frac": by / (ms * 1e-3) / 1e9 / hbm_peak}
+    ach = by / (ms * 1e-3) / 1e9
+    return {"kernel": path, "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
+            "peak_kind": f"of {peak_kind}", "traffic": traffic}
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs.
 
@@ -391,10 +414,9 @@ def main():
                     "frames_per_s": wl.n / (per_path_ms[p] * 1e-3), "algorithmic_bytes": by, "achieved_gbs": gbs,
                     "frac_of_hbm": gbs / peak}
     dominant = max(active, key=lambda p: per_path_ms[p])
-    tr = NCU_TRAFFIC_BYTES_PER_PIXEL.get(dominant)
-    roofline = {"kernel": dominant, "bound": "hbm", "achieved": paths[dominant]["achieved_gbs"], "peak": peak,
-                "unit": "GB/s", "frac": paths[dominant]["frac_of_hbm"], "peak_kind": f"of {peak_kind}",
-                "traffic": None if tr is None else tr * wl.npix}
+    roofline = path_roofline(wl, dominant, per_path_ms[dominant], peak, peak_kind, NCU_TRAFFIC_BYTES_PER_PIXEL.get(dominant))
+    for p in active:
+        paths[p]["roofline"] = path_roofline(wl, p, per_path_ms[p], peak, peak_kind, NCU_TRAFFIC_BYTES_PER_PIXEL.get(p))
 
     cpu = None
     if not args.no_cpu_baseline:

@@ -108,7 +108,8 @@ int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, co
  *   SR_COEF_COMPACT:         w_q = coef_or_sel[n][q][Y][X]  (idx required)
  *   SR_IDX_GLOBAL:           a_q = idx[q], w_q = gamma[q] * coef[n][a_q][Y][X]  (gamma NULL = 1);
  *                            with SR_COEF_COMPACT, w_q = gamma[q] * coef_or_sel[n][q][Y][X]
- * Kept coefficients are used unchanged (no renormalisation).  An idx value >= D
+ * Kept coefficients are used unchanged (no renormalisation).  The s indices of a pixel must be distinct (as
+ * sr_dict_select writes them); repeated indices give an unspecified value for that pixel.  An idx value >= D
  * is the caller's error: that pixel's value is then undefined, but no
  * out-of-range access is made (the value is clamped to D-1).
  */
