@@ -52,16 +52,24 @@ namespace th8 {
 
 } // namespace
 
+// Tile height per mode: 16 rows wherever the shape still leaves the selective pipeline its eight stages (dense and
+// global-subset modes always; the in-kernel selection when the single U buffer it needs fits), else 8 rows.
+static bool tall_tiles(int mode, const void* coef, int coef_dtype, const Problem& pb)
+{
+    if (!th8::is_selective(mode)) return true;
+    return mode == kModeFusedSelect && th16::supported(mode, coef, coef_dtype, pb) && th16::stage_count(mode, pb) >= 8;
+}
+
 bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& pb)
 {
-    return th8::is_selective(mode) ? th8::supported(mode, coef, coef_dtype, pb) : th16::supported(mode, coef, coef_dtype, pb);
+    return tall_tiles(mode, coef, coef_dtype, pb) ? th16::supported(mode, coef, coef_dtype, pb) : th8::supported(mode, coef, coef_dtype, pb);
 }
 
 cudaError_t launch_regress_umma(int mode, const float* lr, const void* coef, const uint8_t* idx, const float* gamma,
                                 const float* dict, float* out, const Problem& pb, cudaStream_t st)
 {
-    return th8::is_selective(mode) ? th8::launch(mode, lr, coef, idx, gamma, dict, out, pb, st)
-                                    : th16::launch(mode, lr, coef, idx, gamma, dict, out, pb, st);
+    return tall_tiles(mode, coef, SR_F16, pb) ? th16::launch(mode, lr, coef, idx, gamma, dict, out, pb, st)
+                                               : th8::launch(mode, lr, coef, idx, gamma, dict, out, pb, st);
 }
 
 } // namespace sr
