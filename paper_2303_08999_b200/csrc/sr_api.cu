@@ -149,8 +149,8 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     else if (flags & SR_COEF_COMPACT) mode = kModeCompact;
     else mode = idx ? kModeIdx : kModeFusedSelect;
     cudaError_t err;
-    const bool idx_pairs_ok = !idx || (flags & SR_IDX_GLOBAL) || ((reinterpret_cast<uintptr_t>(idx) & 1) == 0);   // uchar2 reads
-    if (idx_pairs_ok && umma_supported(mode, coef_or_sel, coef_dtype, pb))
+    const bool idx_vec_ok = !idx || (flags & SR_IDX_GLOBAL) || ((reinterpret_cast<uintptr_t>(idx) & 15) == 0);   // 16-byte reads
+    if (idx_vec_ok && umma_supported(mode, coef_or_sel, coef_dtype, pb))
         err = launch_regress_umma(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
     else
         err = launch_regress_fma(mode, lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, pb, (cudaStream_t)stream);

@@ -105,9 +105,10 @@ select_pair_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
             int ga[S], gb[S];
 #pragma unroll
             for (int i = 0; i < S; ++i) {
-                const int tag = 255 - (l0 + i);
-                ga[i] = (l0 + i < D) ? (int)(((w[i] << 8) & 0x7FFF00u) | (uint32_t)tag) : -1;
-                gb[i] = (l0 + i < D) ? (int)(((w[i] >> 8) & 0x7FFF00u) | (uint32_t)tag) : -1;
+                // key = 0 | magnitude (2 bytes) | tag: one byte permute per pixel out of (signs cleared, tag)
+                const uint32_t tag = (uint32_t)(255 - (l0 + i)), m2 = w[i] & 0x7FFF7FFFu;
+                ga[i] = (l0 + i < D) ? (int)__byte_perm(m2, tag, 0x5104) : -1;
+                gb[i] = (l0 + i < D) ? (int)__byte_perm(m2, tag, 0x5324) : -1;
             }
             sort_desc<S>(ga);
             sort_desc<S>(gb);
