@@ -81,12 +81,14 @@ def load_peaks():
 
 # DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
 # kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": 155.05, "select": 174.6, "compact": None, "fused": 154.8, "global": 17.1}
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": 154.8, "select": 169.3, "compact": None, "fused": 155.0, "global": 17.2}
 
 
-# Half-rate integer / binary16 max-min-compare operations per HR pixel of the two selection kernels (sorting-network
-# merges; counted in the design doc section 5) and the B200 rate of that pipe: 148 SMs x 64 lanes/clk x 1.965 GHz.
-ALU_OPS_PER_PIXEL = {"select": 630.0, "fused": 459.0}
+# Half-rate ALU-pipe lane operations per HR pixel of the two selection kernels (sorting-network max/min plus the
+# logic and address operations that share their pipe; counted in the design doc section 5) and the B200 rate of that
+# pipe: 148 SMs x 64 lanes/clk x 1.965 GHz. The fused kernel works on packed binary16 pairs (two pixels per lane
+# operation): 315 max/min + 36 logic + 40 address operations per pixel, below its HBM time, so it is HBM-bound.
+ALU_OPS_PER_PIXEL = {"select": 630.0, "fused": 391.0}
 ALU_PEAK_GOPS = 148 * 64 * 1.965
 
 

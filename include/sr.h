@@ -34,7 +34,8 @@
  *     reported by sr_device_status (the output of that call is then undefined).
  *   - Alignment: lr, hr/out, dict and gamma 4 bytes; coef/sel their element size
  *     (the tensor-core path additionally needs coef 16-byte aligned and W a
- *     multiple of 8; other inputs take the general path).
+ *     multiple of 8, and for per-pixel idx planes idx 16-byte aligned and W a
+ *     multiple of 16; other inputs take the general path).
  */
 #ifndef SR_H_
 #define SR_H_
@@ -108,6 +109,7 @@ int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, co
  *   SR_COEF_COMPACT:         w_q = coef_or_sel[n][q][Y][X]  (idx required)
  *   SR_IDX_GLOBAL:           a_q = idx[q], w_q = gamma[q] * coef[n][a_q][Y][X]  (gamma NULL = 1);
  *                            with SR_COEF_COMPACT, w_q = gamma[q] * coef_or_sel[n][q][Y][X]
+ * With idx == NULL the coefficients must be finite (the selection multiplies dropped ones by zero).
  * Kept coefficients are used unchanged (no renormalisation).  The s indices of a pixel must be distinct (as
  * sr_dict_select writes them); repeated indices give an unspecified value for that pixel.  An idx value >= D
  * is the caller's error: that pixel's value is then undefined, but no
