@@ -97,18 +97,36 @@ select_pair_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
         int ta[S], tb[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1;
-        for (int l0 = 0; l0 < D; l0 += S) {
+        const uint32_t* wp = reinterpret_cast<const uint32_t*>(cp);      // one word = the pair's coefficients of a plane
+        const int64_t wstride = HW / 2;                                   // words between planes (W is even)
+        int l0 = 0;
+        for (; l0 + S <= D; l0 += S) {                                   // whole groups: no per-key guards
             uint32_t w[S];
 #pragma unroll
-            for (int i = 0; i < S; ++i)
-                w[i] = (l0 + i < D) ? __ldg(reinterpret_cast<const uint32_t*>(cp + (int64_t)(l0 + i) * HW)) : 0u;
+            for (int i = 0; i < S; ++i) w[i] = __ldg(wp + (int64_t)(l0 + i) * wstride);
             int ga[S], gb[S];
 #pragma unroll
             for (int i = 0; i < S; ++i) {
                 // key = 0 | magnitude (2 bytes) | tag: one byte permute per pixel out of (signs cleared, tag)
                 const uint32_t tag = (uint32_t)(255 - (l0 + i)), m2 = w[i] & 0x7FFF7FFFu;
-                ga[i] = (l0 + i < D) ? (int)__byte_perm(m2, tag, 0x5104) : -1;
-                gb[i] = (l0 + i < D) ? (int)__byte_perm(m2, tag, 0x5324) : -1;
+                ga[i] = (int)__byte_perm(m2, tag, 0x5104);
+                gb[i] = (int)__byte_perm(m2, tag, 0x5324);
+            }
+            sort_desc<S>(ga);
+            sort_desc<S>(gb);
+            merge_top<S>(ta, ga);
+            merge_top<S>(tb, gb);
+        }
+        if (l0 < D) {                                                     // last, partial group
+            int ga[S], gb[S];
+#pragma unroll
+            for (int i = 0; i < S; ++i) {
+                ga[i] = gb[i] = -1;
+                if (l0 + i < D) {
+                    const uint32_t tag = (uint32_t)(255 - (l0 + i)), m2 = __ldg(wp + (int64_t)(l0 + i) * wstride) & 0x7FFF7FFFu;
+                    ga[i] = (int)__byte_perm(m2, tag, 0x5104);
+                    gb[i] = (int)__byte_perm(m2, tag, 0x5324);
+                }
             }
             sort_desc<S>(ga);
             sort_desc<S>(gb);
