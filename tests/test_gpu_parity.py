@@ -139,6 +139,13 @@ SEL_CASES = [
     (1, 1, 12, 24, 2, 128, 7, "f16", 16),
     (1, 3, 8, 24, 2, 72, 5, "f16", 20),
     (1, 3, 8, 24, 2, 16, 5, "f16", 16),
+    # widths that are multiples of 16: the index-listed and compact modes take the tensor-core kernel too
+    (1, 3, 24, 64, 2, 72, 5, "f16", 8),
+    (1, 3, 20, 36, 4, 32, 3, "f16", 4),
+    (2, 3, 9, 40, 2, 128, 5, "f16", 8),
+    (1, 3, 10, 24, 2, 20, 5, "f16", 3),
+    (1, 2, 40, 72, 4, 72, 3, "f16", 8),
+    (1, 3, 7, 168, 2, 6, 7, "f16", 6),
 ]
 
 
@@ -183,10 +190,18 @@ def test_selected_with_s_equal_D_is_dense():
     assert max_abs_err(a, oracle.dict_regress_dense(lr, coef, dict_, 2, 5)) <= TOL_F16
 
 
-def test_selected_with_ties():
-    wl = _wl(1, 3, 16, 24, 2, 72, 5, "f16")
+@pytest.mark.parametrize("D,s,w", [(72, 8, 24), (128, 5, 64), (24, 8, 32), (72, 1, 24)])
+def test_selected_with_ties(D, s, w):
+    wl = _wl(1, 3, 16, w, 2, D, 5, "f16")
     lr, dict_, coef = sr_inputs.make_inputs(wl)
     coef = _coarse(coef)
-    want = oracle.dict_regress_selected(lr, coef, None, None, dict_, 2, 5, 8)
-    got = host(sr.sr_dict_regress_selected(dev(lr), dev(coef), None, None, dev(dict_), 2, 5, 8))
+    want = oracle.dict_regress_selected(lr, coef, None, None, dict_, 2, 5, s)
+    got = host(sr.sr_dict_regress_selected(dev(lr), dev(coef), None, None, dev(dict_), 2, 5, s))
+    assert max_abs_err(got, want) <= TOL_F16
+    # the same pixels through explicit index planes (ties resolved by sr_dict_select) and compact values
+    idx, sel = sr.sr_dict_select(dev(coef), s, want_sel=True)
+    np.testing.assert_array_equal(host(idx), oracle.dict_select(coef, s))
+    got = host(sr.sr_dict_regress_selected(dev(lr), dev(coef), idx, None, dev(dict_), 2, 5, s))
+    assert max_abs_err(got, want) <= TOL_F16
+    got = host(sr.sr_dict_regress_selected(dev(lr), sel, idx, None, dev(dict_), 2, 5, s, sr.SR_COEF_COMPACT))
     assert max_abs_err(got, want) <= TOL_F16
