@@ -1,6 +1,5 @@
 """Shape sweep of the regression paths (the cfg4 benchmark configuration): LR 3x360x640, scale in {2,3,4},
-D in {16,32,72,128}, k in {3,5,7}; dense and fused selective (s in {4,8,16}, skipped when s > D or the path is
-not implemented for that s on the tensor cores, where the general kernel runs instead).
+D in {16,32,72,128}, k in {3,5,7}; dense and fused selective (s in {4,8,16}, skipped when s > D).
 
     python -m paper_2303_08999_b200.sweep [--hbm-gbs 6459] [--cfg3]
 

@@ -146,6 +146,10 @@ SEL_CASES = [
     (1, 3, 10, 24, 2, 20, 5, "f16", 3),
     (1, 2, 40, 72, 4, 72, 3, "f16", 8),
     (1, 3, 7, 168, 2, 6, 7, "f16", 6),
+    # 8 < s <= 16: the sixteen-entry list of the in-kernel selection, two rank halves per lane in the listed modes
+    (1, 3, 12, 32, 2, 72, 5, "f16", 12),
+    (1, 3, 12, 64, 4, 128, 3, "f16", 16),
+    (1, 3, 10, 40, 2, 24, 5, "f16", 9),
 ]
 
 
@@ -190,7 +194,7 @@ def test_selected_with_s_equal_D_is_dense():
     assert max_abs_err(a, oracle.dict_regress_dense(lr, coef, dict_, 2, 5)) <= TOL_F16
 
 
-@pytest.mark.parametrize("D,s,w", [(72, 8, 24), (128, 5, 64), (24, 8, 32), (72, 1, 24)])
+@pytest.mark.parametrize("D,s,w", [(72, 8, 24), (128, 5, 64), (24, 8, 32), (72, 1, 24), (72, 13, 32), (40, 16, 24)])
 def test_selected_with_ties(D, s, w):
     wl = _wl(1, 3, 16, w, 2, D, 5, "f16")
     lr, dict_, coef = sr_inputs.make_inputs(wl)
