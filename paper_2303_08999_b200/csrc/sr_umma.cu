@@ -17,7 +17,8 @@
 //
 // Warp roles, dense and global-subset modes (640 threads = five warpgroups; the register file is re-balanced between
 // them with setmaxnreg):
-//   warps 0-3    coefficient producers   full[stage] <- copy arrivals when the data has landed; wait empty[stage]
+//   warps 0-3    coefficient producers (two groups, alternate rows)   full[stage] <- copy arrivals when the data
+//                has landed; wait empty[stage]
 //   warps 4-5    MMA issuers (warp 4 owns TMEM): one thread each, alternate rows, because the issue loop of a
 //                single thread (~600 cycles per row alone, twice that on a busy SM) would otherwise pace the kernel;
 //                acc_full[a], empty[stage] <- tcgen05.commit; wait full[stage] (ready[stage] when selecting), acc_empty[a]
