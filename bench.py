@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1]
 
 One step = one pass of the whole hot path over one frame batch of the workload (default: the
-1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. five library
+1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. six library
 calls on one stream:
+    bicubic    sr_bicubic_upsample                           (stage 1 alone)
     dense      sr_dict_regress_dense                         (up-sample + assemble + filter, fused)
     select     sr_dict_select (indices + selected values)
     compact    sr_dict_regress_selected from those index / value planes
@@ -32,7 +33,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-PATHS = ("dense", "select", "compact", "fused", "global")
+PATHS = ("bicubic", "dense", "select", "compact", "fused", "global")
 METRIC = "HR megapixels/s"
 
 
@@ -42,6 +43,7 @@ def algorithmic_bytes_per_pixel(wl, path: str) -> float:
     io = 4 * wl.c + 4 * wl.c / (wl.scale ** 2)
     s, D = wl.s, wl.D
     return {
+        "bicubic": io,                             # LR read, up-sampled frame written
         "dense": D * cb + io,
         "select": D * cb + s + s * cb,            # read all planes, write uint8 indices and selected values
         "compact": s * (cb + 1) + io,             # read index + value planes
@@ -81,7 +83,7 @@ def load_peaks():
 
 # DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
 # kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"dense": 154.6, "select": 165.9, "compact": 25.9, "fused": 155.2, "global": 17.1}
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.6, "select": 165.9, "compact": 25.9, "fused": 155.2, "global": 17.1}
 
 
 # Half-rate ALU-pipe lane operations per HR pixel of the two selection kernels (sorting-network max/min plus the
@@ -176,11 +178,12 @@ class ClockSampler:
 
 
 def oracle_step(oracle, wl, lr, dict_, coef, S, gamma, rows: int | None, threads: int = 0):
-    """The step's five paths on the CPU oracle, on the top `rows` LR rows of every frame (None = all)."""
+    """The step's six paths on the CPU oracle, on the top `rows` LR rows of every frame (None = all)."""
     if rows is not None and rows < wl.h:
         lr = lr[:, :, :rows].copy()
         coef = coef[:, :, : rows * wl.scale].copy()
     r, k, s = wl.scale, wl.k, wl.s
+    oracle.bicubic_upsample(lr, r, threads=threads)
     oracle.dict_regress_dense(lr, coef, dict_, r, k, flags=oracle.CLAMP01, threads=threads)
     idx, sel = oracle.dict_select(coef, s, want_sel=True, threads=threads)
     sel = sel.astype(coef.dtype)
@@ -207,7 +210,7 @@ def time_oracle(wl, lr, dict_, coef, S, gamma, budget_s: float = 20.0):
         px += oracle_step(oracle, wl, lr[:1], dict_, coef[:1], S, gamma, rows)
     dt = time.perf_counter() - t0
     return {"value": px / dt / 1e6, "unit": METRIC, "cores": oracle.max_threads(), "kind": "oracle",
-            "sample": f"top {rows} of {wl.h} LR rows of one frame, {reps} times ({px} HR pixels), all five paths of a "
+            "sample": f"top {rows} of {wl.h} LR rows of one frame, {reps} times ({px} HR pixels), all six paths of a "
                       f"step, {dt:.2f} s of fp64 CPU work"}
 
 
@@ -236,7 +239,7 @@ def run_reference(args, wl):
         px += oracle_step(oracle, one, lr, dict_, coef, S, gamma, rows)
     dt = time.perf_counter() - t0
     value = px / dt / 1e6
-    sample = f"top {rows} of {wl.h} LR rows of one frame per step, all five paths"
+    sample = f"top {rows} of {wl.h} LR rows of one frame per step, all six paths"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "MP/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -306,7 +309,7 @@ def main():
     for _ in range(nsets):
         sets.append({"lr": h_lr.cuda(non_blocking=True), "coef": h_coef.cuda(non_blocking=True)})
     shape_out = (wl.n, wl.c, wl.H, wl.W)
-    outs = {p: torch.empty(shape_out, dtype=torch.float32, device="cuda") for p in ("dense", "compact", "fused", "global")}
+    outs = {p: torch.empty(shape_out, dtype=torch.float32, device="cuda") for p in ("bicubic", "dense", "compact", "fused", "global")}
     idx = torch.empty((wl.n, wl.s, wl.H, wl.W), dtype=torch.uint8, device="cuda")
     sel = torch.empty((wl.n, wl.s, wl.H, wl.W), dtype=h_coef.dtype, device="cuda")
     flags = sr.SR_CLAMP01
@@ -319,6 +322,9 @@ def main():
                 e = torch.cuda.Event(enable_timing=True)
                 e.record()
                 events.append(e)
+        mark()
+        if "bicubic" in active:
+            sr.sr_bicubic_upsample(bufs["lr"], r, out=outs["bicubic"])
         mark()
         if "dense" in active:
             sr.sr_dict_regress_dense(bufs["lr"], bufs["coef"], d_dict, r, k, flags, out=outs["dense"])
