@@ -46,6 +46,11 @@ def _check_workload(wl, nsamples):
     r, k, s = wl.scale, wl.k, wl.s
     flags = sr.SR_CLAMP01
 
+    up = sr.sr_bicubic_upsample(dlr, r)                      # stage 1 alone: the whole frame against the oracle
+    err = np.abs(host(up).astype(np.float64) - oracle.bicubic_upsample(lr, r)).max()
+    assert err <= 2e-6, f"bicubic {err}"
+    del up
+
     out = sr.sr_dict_regress_dense(dlr, dco, ddi, r, k, flags)
     want = oracle.regress_at("dense", lr, coef, None, None, dict_, samples, r, k, flags=oracle.CLAMP01)
     err = np.abs(_gather(out, samples, wl) - want).max()
@@ -70,6 +75,9 @@ def _check_workload(wl, nsamples):
     out = sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, r, k, s, flags | sr.SR_COEF_COMPACT)
     err = np.abs(_gather(out, samples, wl) - want).max()
     assert err <= TOL_F16, f"compact selected {err}"
+    out = sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, r, k, s, flags)
+    err = np.abs(_gather(out, samples, wl) - want).max()
+    assert err <= TOL_F16, f"index-listed selected {err}"
     del out, idx, sel
 
     S = np.arange(0, wl.D, wl.D // s, dtype=np.uint8)[:s]
