@@ -202,8 +202,8 @@ def time_oracle(wl, lr, dict_, coef, S, gamma, budget_s: float = 20.0):
     dt = time.perf_counter() - t0
     rate = px / dt
     rows = int(max(probe_rows, min(wl.h, budget_s * rate / (wl.W * wl.scale))))
-    # when a whole frame takes less than the budget, the same band is repeated until about 10 s have been spent
-    reps = int(max(1, min(64, (0.5 * budget_s * rate) // max(1, rows * wl.scale * wl.W))))
+    # when a whole frame takes less than the budget, the same band is repeated until about 14 s have been spent
+    reps = int(max(1, min(64, (0.7 * budget_s * rate) // max(1, rows * wl.scale * wl.W))))
     t0 = time.perf_counter()
     px = 0
     for _ in range(reps):
