@@ -61,7 +61,8 @@ namespace th8 {
 static bool tall_tiles(int mode, const void* coef, int coef_dtype, const Problem& pb)
 {
     if (!th8::is_selective(mode)) return true;
-    return th16::supported(mode, coef, coef_dtype, pb) && th16::stage_count(mode, pb) >= 8;
+    // (compact values: nothing streams into the stages, four are enough)
+    return th16::supported(mode, coef, coef_dtype, pb) && th16::stage_count(mode, pb) >= (mode == kModeCompact ? 4 : 8);
 }
 
 bool umma_supported(int mode, const void* coef, int coef_dtype, const Problem& pb)
