@@ -9,6 +9,8 @@
 //   bitonic sequence holding the S best of both), bitonic-merge it back to sorted order (S/2 * log2 S exchanges).
 // Per pixel and plane that is about 8.75 min/max for S = 8 (630 per pixel at D = 72) against 16 for plain insertion.
 // The kernel is bound by the integer ALU rate or by HBM, whichever is slower for the shape.
+// With 16-byte aligned planes the block first stages its 512 pixels x D planes in shared memory (select_tile_kernel)
+// and the threads read their words, and at the end the selected values, from there.
 #include "sr_common.cuh"
 
 namespace sr {
