@@ -81,6 +81,15 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, v
     return ok != 0;
 }
 
+// Whole-warp wait in which every lane tests the barrier itself (one shared-memory round trip when the phase is
+// already complete, against three for mbar_wait_warp: lane 0's test, the shuffle, the other lanes' test). `seen`:
+// the result of a test issued earlier (true = the phase was already complete then, nothing left to do).
+__device__ __forceinline__ bool mbar_wait_lanes(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool seen)
+{
+    if (__all_sync(0xffffffffu, seen)) return true;
+    return mbar_wait(bar, parity, abort_flag);
+}
+
 // ---- proxies / fences ----------------------------------------------------------------------------------------------
 
 // Makes shared-memory writes of the generic proxy visible to the async proxy (TMA, tcgen05.mma operands).
