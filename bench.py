@@ -83,7 +83,7 @@ def load_peaks():
 
 # DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
 # kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.6, "select": 161.7, "compact": 25.9, "fused": 155.2, "global": 17.1}
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.2, "select": 161.7, "compact": 25.7, "fused": 154.3, "global": 17.0}
 
 
 # Half-rate ALU-pipe lane operations per HR pixel of the two selection kernels (sorting-network max/min plus the
