@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "sr_ref.cpp")
 _LIB = os.path.join(_HERE, "libsr_ref.so")
 
 F32, F16 = 0, 1
-CLAMP01, IDX_GLOBAL, COEF_COMPACT = 1, 2, 4
+CLAMP01, IDX_GLOBAL, COEF_COMPACT, UPSAMPLE_BILINEAR = 1, 2, 4, 8
 
 _lib = None
 
@@ -36,13 +36,14 @@ def _load():
         L = ctypes.CDLL(build())
         vp, i32, i64, u32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint
         L.sr_ref_bicubic_upsample.argtypes = [vp, vp] + [i32] * 6
+        L.sr_ref_bilinear_upsample.argtypes = [vp, vp] + [i32] * 6
         L.sr_ref_dict_regress_dense.argtypes = [vp, vp, i32, vp, vp] + [i32] * 7 + [u32, i32]
         L.sr_ref_dict_select.argtypes = [vp, i32, vp, vp] + [i32] * 6
         L.sr_ref_dict_regress_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp] + [i32] * 8 + [u32, i32]
         L.sr_ref_regress_at.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, i64, vp] + [i32] * 8 + [u32, i32]
         L.sr_ref_dict_select_at.argtypes = [vp, i32, vp, i64, vp] + [i32] * 6
         L.sr_ref_max_threads.argtypes = []
-        for f in (L.sr_ref_bicubic_upsample, L.sr_ref_dict_regress_dense, L.sr_ref_dict_select,
+        for f in (L.sr_ref_bicubic_upsample, L.sr_ref_bilinear_upsample, L.sr_ref_dict_regress_dense, L.sr_ref_dict_select,
                   L.sr_ref_dict_regress_selected, L.sr_ref_regress_at, L.sr_ref_dict_select_at, L.sr_ref_max_threads):
             f.restype = i32
         _lib = L
@@ -76,6 +77,14 @@ def bicubic_upsample(lr: np.ndarray, scale: int, threads: int = 0) -> np.ndarray
     n, c, h, w = lr.shape
     out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
     _check(_load().sr_ref_bicubic_upsample(lr.ctypes.data, out.ctypes.data, n, c, h, w, scale, threads), "bicubic")
+    return out
+
+
+def bilinear_upsample(lr: np.ndarray, scale: int, threads: int = 0) -> np.ndarray:
+    lr = _c(lr, np.float32)
+    n, c, h, w = lr.shape
+    out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_bilinear_upsample(lr.ctypes.data, out.ctypes.data, n, c, h, w, scale, threads), "bilinear")
     return out
 
 

@@ -19,8 +19,10 @@
  * Parity pins (tests/test_oracle_pins.py): closed-form bicubic weights, a library
  * bicubic resize, a library cross-correlation on the replicate-padded image, a
  * hand-worked 4x4 example, delta-atom / constant-image / linearity / s = D /
- * prefix / permutation identities, and a brute-force sort for the selection.
- * No function here is parity-unpinned.
+ * prefix / permutation identities, and a brute-force sort for the selection;
+ * for the bilinear variant of stage 1a a library bilinear resize, closed-form
+ * weights, exact reproduction of affine images away from the border and the
+ * delta-atom identity.  No function here is parity-unpinned.
  */
 #include <algorithm>
 #include <cmath>
@@ -35,7 +37,7 @@
 namespace {
 
 enum { REF_F32 = 0, REF_F16 = 1 };
-enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u };
+enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u, REF_UPSAMPLE_BILINEAR = 8u };
 enum { REF_OK = 0, REF_ERR_NULL = 1, REF_ERR_SHAPE = 2, REF_ERR_UNSUPPORTED = 3 };
 
 struct Dims {
@@ -201,6 +203,30 @@ void gather_selected(const Dims& d, const void* coef_or_sel, int dtype, const ui
     }
 }
 
+/*
+ * Stage 1a as the paper words it (Section II-A: "bilinear up-sampling is adopted"): the value at the same
+ * half-pixel sample point src = (X + 1/2)/r - 1/2, interpolated linearly between the two nearest LR samples
+ * per axis, indices clamped to the image.
+ */
+double bilinear_at(const float* plane, int h, int w, int r, int Y, int X)
+{
+    const double sy = (Y + 0.5) / r - 0.5;
+    const double sx = (X + 0.5) / r - 0.5;
+    const int iy = (int)std::floor(sy);
+    const int ix = (int)std::floor(sx);
+    const double ty = sy - iy, tx = sx - ix;
+    const int y0 = clampi(iy, 0, h - 1), y1 = clampi(iy + 1, 0, h - 1);
+    const int x0 = clampi(ix, 0, w - 1), x1 = clampi(ix + 1, 0, w - 1);
+    const double top = (1.0 - tx) * (double)plane[(int64_t)y0 * w + x0] + tx * (double)plane[(int64_t)y0 * w + x1];
+    const double bot = (1.0 - tx) * (double)plane[(int64_t)y1 * w + x0] + tx * (double)plane[(int64_t)y1 * w + x1];
+    return (1.0 - ty) * top + ty * bot;
+}
+
+double upsample_at(const float* plane, int h, int w, int r, int Y, int X, unsigned flags)
+{
+    return (flags & REF_UPSAMPLE_BILINEAR) ? bilinear_at(plane, h, w, r, Y, X) : bicubic_at(plane, h, w, r, Y, X);
+}
+
 void set_threads(int threads)
 {
 #ifdef _OPENMP
@@ -211,7 +237,7 @@ void set_threads(int threads)
 }
 
 /* U for the whole batch, [n][c][H][W] */
-void upsample_all(const float* lr, const Dims& d, std::vector<double>& U)
+void upsample_all(const float* lr, const Dims& d, std::vector<double>& U, unsigned flags)
 {
     const int H = d.H(), W = d.W();
     U.resize((size_t)d.n * d.c * H * W);
@@ -221,7 +247,7 @@ void upsample_all(const float* lr, const Dims& d, std::vector<double>& U)
         for (int Y = 0; Y < H; ++Y) {
             const float* src = lr + pl * (int64_t)d.h * d.w;
             double* dst = U.data() + (pl * H + Y) * (int64_t)W;
-            for (int X = 0; X < W; ++X) dst[X] = bicubic_at(src, d.h, d.w, d.r, Y, X);
+            for (int X = 0; X < W; ++X) dst[X] = upsample_at(src, d.h, d.w, d.r, Y, X, flags);
         }
 }
 
@@ -237,7 +263,20 @@ int sr_ref_bicubic_upsample(const float* lr, double* hr, int n, int c, int h, in
     if (int e = check_dims(d)) return e;
     set_threads(threads);
     std::vector<double> U;
-    upsample_all(lr, d, U);
+    upsample_all(lr, d, U, 0u);
+    std::memcpy(hr, U.data(), U.size() * sizeof(double));
+    return REF_OK;
+}
+
+/* Stage 1a alone, bilinear form: hr[n][c][H][W] (fp64) from lr[n][c][h][w] (fp32). */
+int sr_ref_bilinear_upsample(const float* lr, double* hr, int n, int c, int h, int w, int r, int threads)
+{
+    Dims d{n, c, h, w, r, 1, 1};
+    if (!lr || !hr) return REF_ERR_NULL;
+    if (int e = check_dims(d)) return e;
+    set_threads(threads);
+    std::vector<double> U;
+    upsample_all(lr, d, U, REF_UPSAMPLE_BILINEAR);
     std::memcpy(hr, U.data(), U.size() * sizeof(double));
     return REF_OK;
 }
@@ -253,7 +292,7 @@ int sr_ref_dict_regress_dense(const float* lr, const void* coef, int coef_dtype,
     const int H = d.H(), W = d.W();
     const int64_t HW = (int64_t)H * W;
     std::vector<double> U;
-    upsample_all(lr, d, U);
+    upsample_all(lr, d, U, flags);
     std::vector<int> atoms((size_t)L);
     for (int l = 0; l < L; ++l) atoms[(size_t)l] = l;
     for (int f = 0; f < n; ++f) {
@@ -322,7 +361,7 @@ int sr_ref_dict_regress_selected(const float* lr, const void* coef_or_sel, int c
     const int H = d.H(), W = d.W();
     const int64_t HW = (int64_t)H * W;
     std::vector<double> U;
-    upsample_all(lr, d, U);
+    upsample_all(lr, d, U, flags);
     for (int f = 0; f < n; ++f) {
 #pragma omp parallel for schedule(static)
         for (int Y = 0; Y < H; ++Y) {
@@ -376,7 +415,7 @@ int sr_ref_regress_at(int mode, const float* lr, const void* coef_or_sel, int co
             gather_selected(d, coef_or_sel, coef_dtype, idx, gamma, s, flags, f, pix, atoms.data(), wts.data());
         }
         auto patch = [&](int ch, int yy, int xx) {
-            return bicubic_at(lr + ((int64_t)f * c + ch) * d.h * d.w, d.h, d.w, d.r, yy, xx);
+            return upsample_at(lr + ((int64_t)f * c + ch) * d.h * d.w, d.h, d.w, d.r, yy, xx, flags);
         };
         regress_pixel(d, dict, s, atoms.data(), wts.data(), Y, X, flags, patch, out + i * c);
     }
