@@ -58,7 +58,9 @@ enum { SR_F32 = 0, SR_F16 = 1 }; /* coefficient storage type */
 enum {
     SR_CLAMP01 = 1u,      /* clamp the output to [0,1] as the last step                                */
     SR_IDX_GLOBAL = 2u,   /* idx[s] (+ gamma[s]) is one atom subset for every pixel                    */
-    SR_COEF_COMPACT = 4u  /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
+    SR_COEF_COMPACT = 4u, /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
+    SR_UPSAMPLE_BILINEAR = 8u /* stage 1 interpolates linearly between the two nearest LR samples per axis
+                                 (the paper's wording, Section II-A) instead of the bicubic kernel            */
 };
 
 enum {
@@ -80,10 +82,19 @@ enum {
 int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream);
 
 /*
+ * Stage 1 alone in the form the paper's text names (Section II-A, "bilinear
+ * up-sampling is adopted"): the same half-pixel sample point, linear
+ * interpolation between the two nearest LR samples per axis, indices clamped
+ * to the image.  lr must be finite (the two outer taps of the shared four-tap
+ * window are multiplied by zero).  d->k and d->D are ignored.
+ */
+int sr_bilinear_upsample(const float* lr, float* hr, const sr_dims* d, void* stream);
+
+/*
  * Stages 1, 3 and 4 with every atom (Eq. 2: y_i = F_i B_i^T with F_i = Phi_i D;
  * image form Eq. 3): out[n][c][Y][X] = sum_j (sum_l coef[n][l][Y][X] * dict[l][j]) * B_c[j],
  * patch positions clamped to the HR image (edge replicate).  fp32 accumulation.
- * flags: SR_CLAMP01 or 0.
+ * flags: any of SR_CLAMP01, SR_UPSAMPLE_BILINEAR.
  */
 int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out,
                           const sr_dims* d, uint32_t flags, void* stream);
@@ -109,6 +120,7 @@ int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, co
  *   SR_COEF_COMPACT:         w_q = coef_or_sel[n][q][Y][X]  (idx required)
  *   SR_IDX_GLOBAL:           a_q = idx[q], w_q = gamma[q] * coef[n][a_q][Y][X]  (gamma NULL = 1);
  *                            with SR_COEF_COMPACT, w_q = gamma[q] * coef_or_sel[n][q][Y][X]
+ * SR_CLAMP01 and SR_UPSAMPLE_BILINEAR may be added to any of these.
  * With idx == NULL the coefficients must be finite (the selection multiplies dropped ones by zero).
  * Kept coefficients are used unchanged (no renormalisation).  The s indices of a pixel must be distinct (as
  * sr_dict_select writes them); repeated indices give an unspecified value for that pixel.  An idx value >= D

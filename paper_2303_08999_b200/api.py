@@ -16,10 +16,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsr.so")
 
 SR_F32, SR_F16 = 0, 1
-SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT = 1, 2, 4
+SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR = 1, 2, 4, 8
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
 
-EXPORTS = ("sr_bicubic_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
+EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
            "sr_status_string", "sr_device_status", "sr_launch_count")
 
 
@@ -46,6 +46,7 @@ def load_library() -> ctypes.CDLL:
         vp, i32, u32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint32
         dp = ctypes.POINTER(sr_dims)
         lib.sr_bicubic_upsample.argtypes = [vp, vp, dp, vp]
+        lib.sr_bilinear_upsample.argtypes = [vp, vp, dp, vp]
         lib.sr_dict_regress_dense.argtypes = [vp, vp, i32, vp, vp, dp, u32, vp]
         lib.sr_dict_select.argtypes = [vp, i32, vp, vp, dp, i32, u32, vp]
         lib.sr_dict_regress_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp, dp, i32, u32, vp]
@@ -91,7 +92,7 @@ def _check(status: int, what: str):
         raise SrError(status, what)
 
 
-def sr_bicubic_upsample(lr: torch.Tensor, scale: int, out: torch.Tensor | None = None) -> torch.Tensor:
+def _upsample(name: str, lr: torch.Tensor, scale: int, out: torch.Tensor | None) -> torch.Tensor:
     lr = _dev(lr, torch.float32, "lr")
     n, c, h, w = lr.shape
     if out is None:
@@ -99,8 +100,16 @@ def sr_bicubic_upsample(lr: torch.Tensor, scale: int, out: torch.Tensor | None =
     _dev(out, torch.float32, "out")
     assert out.shape == (n, c, h * scale, w * scale)
     d = sr_dims(n, c, h, w, scale, 1, 1)
-    _check(load_library().sr_bicubic_upsample(_ptr(lr), _ptr(out), ctypes.byref(d), _stream()), "sr_bicubic_upsample")
+    _check(getattr(load_library(), name)(_ptr(lr), _ptr(out), ctypes.byref(d), _stream()), name)
     return out
+
+
+def sr_bicubic_upsample(lr: torch.Tensor, scale: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    return _upsample("sr_bicubic_upsample", lr, scale, out)
+
+
+def sr_bilinear_upsample(lr: torch.Tensor, scale: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    return _upsample("sr_bilinear_upsample", lr, scale, out)
 
 
 def sr_dict_regress_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, out=None) -> torch.Tensor:

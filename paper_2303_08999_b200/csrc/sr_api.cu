@@ -29,7 +29,8 @@ int* device_status_word()
 
 // Keys cubic-convolution weights (a = -0.75) for every phase of an integer scale, computed in
 // double and rounded once. src = (X + 1/2)/r - 1/2 = (2X + 1 - r) / (2r) in exact integers.
-BicubicPhases make_phases(int r)
+// `bilinear`: the same four-tap window with weights (0, 1 - t, t, 0), so every kernel serves both forms.
+BicubicPhases make_phases(int r, bool bilinear)
 {
     BicubicPhases ph{};
     const double A = -0.75;
@@ -39,10 +40,10 @@ BicubicPhases make_phases(int r)
         const double t = (double)(num - fl * 2 * r) / (double)(2 * r);
         auto inner = [&](double z) { return ((A + 2.0) * z - (A + 3.0)) * z * z + 1.0; };
         auto outer = [&](double z) { return ((A * z - 5.0 * A) * z + 8.0 * A) * z - 4.0 * A; };
-        ph.w[p][0] = (float)outer(t + 1.0);
-        ph.w[p][1] = (float)inner(t);
-        ph.w[p][2] = (float)inner(1.0 - t);
-        ph.w[p][3] = (float)outer(2.0 - t);
+        ph.w[p][0] = bilinear ? 0.f : (float)outer(t + 1.0);
+        ph.w[p][1] = bilinear ? (float)(1.0 - t) : (float)inner(t);
+        ph.w[p][2] = bilinear ? (float)t : (float)inner(1.0 - t);
+        ph.w[p][3] = bilinear ? 0.f : (float)outer(2.0 - t);
         ph.base[p] = fl - 1;
     }
     return ph;
@@ -72,7 +73,7 @@ static Problem make_problem(const sr_dims* d, int s, uint32_t flags)
     pb.n = d->n; pb.c = d->c; pb.h = d->h; pb.w = d->w; pb.r = d->scale; pb.k = d->k; pb.D = d->D;
     pb.H = d->h * d->scale; pb.W = d->w * d->scale;
     pb.s = s; pb.flags = flags;
-    pb.ph = make_phases(d->scale);
+    pb.ph = make_phases(d->scale, (flags & SR_UPSAMPLE_BILINEAR) != 0);
     return pb;
 }
 
@@ -84,15 +85,25 @@ using namespace sr;
 
 extern "C" {
 
-int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream)
+static int upsample_alone(const float* lr, float* hr, const sr_dims* d, uint32_t flags, void* stream)
 {
     if (!lr || !hr || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, false)) return e;
     if (!aligned(lr, 4) || !aligned(hr, 4)) return SR_ERR_ALIGN;
     sr_dims dd = *d;
     dd.k = 1; dd.D = 1;
-    const Problem pb = make_problem(&dd, 1, 0);
+    const Problem pb = make_problem(&dd, 1, flags);
     return launch_bicubic(lr, hr, pb, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream)
+{
+    return upsample_alone(lr, hr, d, 0u, stream);
+}
+
+int sr_bilinear_upsample(const float* lr, float* hr, const sr_dims* d, void* stream)
+{
+    return upsample_alone(lr, hr, d, SR_UPSAMPLE_BILINEAR, stream);
 }
 
 int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out,
@@ -101,7 +112,7 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)SR_CLAMP01) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR)) return SR_ERR_UNSUPPORTED;
     if (!aligned(lr, 4) || !aligned(out, 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const Problem pb = make_problem(d, d->D, flags);
@@ -136,7 +147,7 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;

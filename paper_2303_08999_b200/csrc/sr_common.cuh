@@ -12,7 +12,8 @@ namespace sr {
 constexpr int kMaxScale = 8;
 constexpr int kMaxK = 9;
 
-// Per-phase bicubic taps of one axis (Keys cubic convolution, a = -0.75, half-pixel centres).
+// Per-phase taps of one axis of the up-sampling (Keys cubic convolution, a = -0.75, half-pixel centres; or the
+// bilinear pair in the two middle taps).
 // HR index X = q*scale + phase reads LR indices q + base[phase] + {0,1,2,3}, each clamped to the image.
 struct BicubicPhases {
     float w[kMaxScale][4];
@@ -36,7 +37,7 @@ enum RegressMode {
     kModeFusedSelect = 4  // top-s chosen inside the kernel from [n][D][H][W]
 };
 
-BicubicPhases make_phases(int scale);
+BicubicPhases make_phases(int scale, bool bilinear);
 
 // Address of the per-device status word (device memory; 0 = ok). Returns nullptr on a CUDA error.
 int* device_status_word();

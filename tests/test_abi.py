@@ -66,6 +66,13 @@ def test_validation_errors_come_back_before_any_launch(lib):
     assert lib.sr_bicubic_upsample(None, FAKE, ctypes.byref(_dims()), None) == api.SR_ERR_NULL
     assert lib.sr_bicubic_upsample(FAKE, FAKE + 2, ctypes.byref(_dims()), None) == api.SR_ERR_ALIGN
     assert lib.sr_bicubic_upsample(FAKE, FAKE, ctypes.byref(_dims(scale=12)), None) == api.SR_ERR_UNSUPPORTED
+    assert lib.sr_bilinear_upsample(None, FAKE, ctypes.byref(_dims()), None) == api.SR_ERR_NULL
+    assert lib.sr_bilinear_upsample(FAKE + 1, FAKE, ctypes.byref(_dims()), None) == api.SR_ERR_ALIGN
+    assert lib.sr_bilinear_upsample(FAKE, FAKE, ctypes.byref(_dims(scale=0)), None) == api.SR_ERR_UNSUPPORTED
+    # the up-sampling variant is a legal flag of the regression calls: validation goes on to the next check
+    assert dense(_dims(k=4), flags=api.SR_UPSAMPLE_BILINEAR) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(), flags=api.SR_UPSAMPLE_BILINEAR | api.SR_CLAMP01, coef=FAKE + 1) == api.SR_ERR_ALIGN
+    assert dense(_dims(), flags=16) == api.SR_ERR_UNSUPPORTED
 
     select = lambda d, s, flags=0, idx=FAKE: lib.sr_dict_select(FAKE, api.SR_F16, idx, None, ctypes.byref(d), s, flags, None)
     assert select(_dims(), 0) == api.SR_ERR_SHAPE
@@ -87,3 +94,5 @@ def test_binding_refuses_cpu_tensors():
     import torch
     with pytest.raises(TypeError):
         sr.sr_bicubic_upsample(torch.zeros(1, 1, 2, 2), 2)
+    with pytest.raises(TypeError):
+        sr.sr_bilinear_upsample(torch.zeros(1, 1, 2, 2), 2)
