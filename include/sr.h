@@ -27,7 +27,10 @@
  *     the caller must free and keeps no reference after the call's work has
  *     run.  Calls are asynchronous on `stream` and never synchronise the host;
  *     buffers must stay valid until the stream reaches the kernels.  `out`
- *     must not alias an input.
+ *     must not alias an input.  Because of this a sequence of calls can be
+ *     recorded into a CUDA graph and replayed; make one ordinary call of each
+ *     kind on the device first (the first launch of a kernel there looks up
+ *     the status word and sets the kernel's shared-memory limit).
  *   - Errors: every call returns an sr status.  Validation failures return
  *     before anything is launched and write nothing.  Nothing throws, aborts or
  *     prints.  A device-side wait that ran out of its iteration limit is
