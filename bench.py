@@ -87,7 +87,8 @@ NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.2, "select": 161.7,
 
 
 # Half-rate ALU-pipe lane operations per HR pixel of the two selection kernels (sorting-network max/min plus the
-# logic and address operations that share their pipe; counted in the design doc section 5) and the B200 rate of that
+# logic and address operations that share their pipe, counted from the networks in csrc/sr_select.cu and the select
+# role of csrc/sr_umma_impl.inc) and the B200 rate of that
 # pipe: 148 SMs x 64 lanes/clk x 1.965 GHz. The fused kernel works on packed binary16 pairs (two pixels per lane
 # operation): 315 max/min + 36 logic + 40 address operations per pixel, below its HBM time, so it is HBM-bound.
 ALU_OPS_PER_PIXEL = {"select": 630.0, "fused": 391.0}
