@@ -14,7 +14,7 @@
  *     as void* (NULL = the legacy default stream).  `d` is a HOST pointer.
  *   - Layouts, all contiguous, row-major, innermost index last:
  *       lr        [n][c][h][w]           fp32   LR image
- *       hr / out  [n][c][H][W]           fp32   H = h*scale, W = w*scale
+ *       hr / out  [n][c][H][W]           fp32   H = h*scale, W = w*scale (out: binary16 with SR_OUT_F16)
  *       coef      [n][D][H][W]           fp32 or binary16 (SR_F32 / SR_F16); one set per
  *                                        frame, shared by the c channels
  *       dict      [D][k*k]               fp32, tap j = a*k + b (a = row) multiplies
@@ -62,8 +62,10 @@ enum {
     SR_CLAMP01 = 1u,      /* clamp the output to [0,1] as the last step                                */
     SR_IDX_GLOBAL = 2u,   /* idx[s] (+ gamma[s]) is one atom subset for every pixel                    */
     SR_COEF_COMPACT = 4u, /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
-    SR_UPSAMPLE_BILINEAR = 8u /* stage 1 interpolates linearly between the two nearest LR samples per axis
-                                 (the paper's wording, Section II-A) instead of the bicubic kernel            */
+    SR_UPSAMPLE_BILINEAR = 8u, /* stage 1 interpolates linearly between the two nearest LR samples per axis
+                                  (the paper's wording, Section II-A) instead of the bicubic kernel           */
+    SR_OUT_F16 = 16u           /* regression calls: `out` is binary16 [n][c][H][W]; the fp32 result is rounded
+                                  to nearest as it is stored (halves the output traffic).  2-byte alignment.  */
 };
 
 enum {
@@ -97,7 +99,7 @@ int sr_bilinear_upsample(const float* lr, float* hr, const sr_dims* d, void* str
  * Stages 1, 3 and 4 with every atom (Eq. 2: y_i = F_i B_i^T with F_i = Phi_i D;
  * image form Eq. 3): out[n][c][Y][X] = sum_j (sum_l coef[n][l][Y][X] * dict[l][j]) * B_c[j],
  * patch positions clamped to the HR image (edge replicate).  fp32 accumulation.
- * flags: any of SR_CLAMP01, SR_UPSAMPLE_BILINEAR.
+ * flags: any of SR_CLAMP01, SR_UPSAMPLE_BILINEAR, SR_OUT_F16 (`out` then points at binary16 elements).
  */
 int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out,
                           const sr_dims* d, uint32_t flags, void* stream);
@@ -123,7 +125,7 @@ int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, co
  *   SR_COEF_COMPACT:         w_q = coef_or_sel[n][q][Y][X]  (idx required)
  *   SR_IDX_GLOBAL:           a_q = idx[q], w_q = gamma[q] * coef[n][a_q][Y][X]  (gamma NULL = 1);
  *                            with SR_COEF_COMPACT, w_q = gamma[q] * coef_or_sel[n][q][Y][X]
- * SR_CLAMP01 and SR_UPSAMPLE_BILINEAR may be added to any of these.
+ * SR_CLAMP01, SR_UPSAMPLE_BILINEAR and SR_OUT_F16 may be added to any of these.
  * With idx == NULL the coefficients must be finite (the selection multiplies dropped ones by zero).
  * Kept coefficients are used unchanged (no renormalisation).  The s indices of a pixel must be distinct (as
  * sr_dict_select writes them); repeated indices give an unspecified value for that pixel.  An idx value >= D

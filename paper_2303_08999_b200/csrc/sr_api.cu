@@ -112,8 +112,8 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const Problem pb = make_problem(d, d->D, flags);
     cudaError_t err;
@@ -147,11 +147,11 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
+    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
         !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const Problem pb = make_problem(d, s, flags);

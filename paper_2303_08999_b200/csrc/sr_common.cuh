@@ -55,6 +55,19 @@ cudaError_t launch_select(const void* coef, int coef_dtype, uint8_t* idx, void* 
 
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v, lo), hi); }
 
+// The fp32 result as it is stored: unchanged, or rounded to nearest binary16 (SR_OUT_F16).
+template <typename OutT> __device__ __forceinline__ OutT to_out(float v);
+template <> __device__ __forceinline__ float to_out<float>(float v) { return v; }
+template <> __device__ __forceinline__ __half to_out<__half>(float v) { return __float2half_rn(v); }
+
+// Output element i of a frame buffer that holds fp32 or (f16) binary16 values; for kernels that are not tight on
+// registers and take the output type at run time.
+__device__ __forceinline__ void store_out(float* out, int64_t i, float v, bool f16)
+{
+    if (f16) reinterpret_cast<__half*>(out)[i] = __float2half_rn(v);
+    else out[i] = v;
+}
+
 __device__ __forceinline__ float load_coef(const float* p, int64_t i) { return __ldg(p + i); }
 __device__ __forceinline__ float load_coef(const __half* p, int64_t i) { return __half2float(__ldg(p + i)); }
 

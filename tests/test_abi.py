@@ -72,7 +72,12 @@ def test_validation_errors_come_back_before_any_launch(lib):
     # the up-sampling variant is a legal flag of the regression calls: validation goes on to the next check
     assert dense(_dims(k=4), flags=api.SR_UPSAMPLE_BILINEAR) == api.SR_ERR_UNSUPPORTED
     assert dense(_dims(), flags=api.SR_UPSAMPLE_BILINEAR | api.SR_CLAMP01, coef=FAKE + 1) == api.SR_ERR_ALIGN
-    assert dense(_dims(), flags=16) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(), flags=32) == api.SR_ERR_UNSUPPORTED
+    # binary16 output: `out` needs 2-byte alignment only (FAKE + 2 passes this check and fails the next one)
+    out_at = lambda out, flags: lib.sr_dict_regress_dense(FAKE, FAKE + 1, api.SR_F16, FAKE, out, ctypes.byref(_dims()), flags, None)
+    assert lib.sr_dict_regress_dense(FAKE, FAKE, api.SR_F16, FAKE, FAKE + 2, ctypes.byref(_dims()), 0, None) == api.SR_ERR_ALIGN
+    assert lib.sr_dict_regress_dense(FAKE, FAKE, api.SR_F16, FAKE, FAKE + 1, ctypes.byref(_dims()), api.SR_OUT_F16, None) == api.SR_ERR_ALIGN
+    assert out_at(FAKE + 2, api.SR_OUT_F16) == api.SR_ERR_ALIGN      # from the odd coefficient pointer, not from `out`
 
     select = lambda d, s, flags=0, idx=FAKE: lib.sr_dict_select(FAKE, api.SR_F16, idx, None, ctypes.byref(d), s, flags, None)
     assert select(_dims(), 0) == api.SR_ERR_SHAPE
