@@ -39,6 +39,13 @@
  *     (the tensor-core path additionally needs coef 16-byte aligned and W a
  *     multiple of 8, and for per-pixel idx planes idx 16-byte aligned and W a
  *     multiple of 16; other inputs take the general path).
+ *   - Value ranges on the tensor-core path (binary16 coefficients, aligned as above, k <= 7, c <= 4): the fp32
+ *     dictionary is held as the sum of two binary16 numbers, so every tap (times gamma, in the global-subset mode)
+ *     must satisfy |tap| < 65504; taps below 2^-14 in magnitude keep an absolute precision of 2^-25 instead of 22
+ *     significant bits.  Coefficients must be finite: the kernel pads the atom count to a multiple of 16 with
+ *     neighbouring staged data times zero dictionary rows, and the in-call selection multiplies dropped
+ *     coefficients by zero, so one Inf or NaN coefficient makes the outputs of its 128-pixel row segment
+ *     unspecified.  The general path has neither restriction.
  */
 #ifndef SR_H_
 #define SR_H_
@@ -63,7 +70,7 @@ enum {
     SR_IDX_GLOBAL = 2u,   /* idx[s] (+ gamma[s]) is one atom subset for every pixel                    */
     SR_COEF_COMPACT = 4u, /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
     SR_UPSAMPLE_BILINEAR = 8u, /* stage 1 interpolates linearly between the two nearest LR samples per axis
-                                  (the paper's wording, Section II-A) instead of the bicubic kernel           */
+                                  (the interpolation Section II-A names) instead of the bicubic kernel        */
     SR_OUT_F16 = 16u           /* regression calls: `out` is binary16 [n][c][H][W]; the fp32 result is rounded
                                   to nearest as it is stored (halves the output traffic).  2-byte alignment.  */
 };
@@ -79,7 +86,7 @@ enum {
 };
 
 /*
- * Stage 1 alone (Section II-A, "the LR input is up-sampled"): hr = bicubic(lr).
+ * Stage 1 alone (Section II-A, the up-sampling that feeds the patch matrix B): hr = bicubic(lr).
  * Keys cubic convolution with a = -0.75, half-pixel centres
  * (src = (X + 1/2)/scale - 1/2), tap indices clamped to the image; the result
  * is not clamped.  d->k and d->D are ignored.
@@ -87,8 +94,8 @@ enum {
 int sr_bicubic_upsample(const float* lr, float* hr, const sr_dims* d, void* stream);
 
 /*
- * Stage 1 alone in the form the paper's text names (Section II-A, "bilinear
- * up-sampling is adopted"): the same half-pixel sample point, linear
+ * Stage 1 alone with the interpolation the paper's text names for stage 1
+ * (Section II-A: bilinear): the same half-pixel sample point, linear
  * interpolation between the two nearest LR samples per axis, indices clamped
  * to the image.  lr must be finite (the two outer taps of the shared four-tap
  * window are multiplied by zero).  d->k and d->D are ignored.
@@ -145,6 +152,23 @@ const char* sr_status_string(int status);
  * SR_ERR_NULL or SR_ERR_CUDA.
  */
 int sr_device_status(void* stream, int* out_status);
+
+/*
+ * Cycle budget of every device-side wait (mbarrier waits for copies, tensor-core results and tile hand-overs) in
+ * the launches that follow, process-wide; the default is 2^31 SM cycles, about a second.  A wait that runs out
+ * makes its thread block stop, wait briefly for its copies and tensor-core operations in flight, free its tensor
+ * memory and return; sr_device_status then reports SR_ERR_TIMEOUT and the call's output is undefined.  Returns the
+ * previous budget; cycles < 1 changes nothing.  Failure handling of this library; the paper has no counterpart.
+ */
+int64_t sr_set_wait_limit(int64_t cycles);
+
+/*
+ * Test hook for the failure path, host-side injection: each of the next `launches` launches of the tensor-core
+ * regression kernel leaves out one barrier arrival in its first thread block, so that one of its waits runs out
+ * (set a small budget with sr_set_wait_limit first).  Nothing faults or spins without bound: the block gives up
+ * as described above.  0 disarms.  Returns SR_OK, or SR_ERR_SHAPE for a negative count.  The paper has no counterpart.
+ */
+int sr_test_lose_arrival(int launches);
 
 /*
  * Number of kernels this library has launched in this process so far (all devices, all streams).

@@ -14,7 +14,8 @@
  * [n][L][H][W]; B_i the k x k patch of the up-sampled image U centred at HR
  * pixel i; F_i = Phi_i D (Eq. 2, right half; Eq. 3 image form) and
  * y_i = F_i B_i^T (Eq. 2, left half), pairing taps with the same index
- * ("Hadamard product ... reducesum", Section III-B).
+ * (Section III-B describes the filtering as an element-wise product of the two
+ * operands summed over the k^2 channels: no flip).
  *
  * Parity pins (tests/test_oracle_pins.py): closed-form bicubic weights, a library
  * bicubic resize, a library cross-correlation on the replicate-padded image, a
@@ -204,7 +205,7 @@ void gather_selected(const Dims& d, const void* coef_or_sel, int dtype, const ui
 }
 
 /*
- * Stage 1a as the paper words it (Section II-A: "bilinear up-sampling is adopted"): the value at the same
+ * Stage 1a with the interpolation the paper's text names (Section II-A: bilinear): the value at the same
  * half-pixel sample point src = (X + 1/2)/r - 1/2, interpolated linearly between the two nearest LR samples
  * per axis, indices clamped to the image.
  */

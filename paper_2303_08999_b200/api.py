@@ -20,7 +20,7 @@ SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16 = 1
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
-           "sr_status_string", "sr_device_status", "sr_launch_count")
+           "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival")
 
 
 class sr_dims(ctypes.Structure):
@@ -55,6 +55,9 @@ def load_library() -> ctypes.CDLL:
             getattr(lib, name).restype = i32
         lib.sr_launch_count.argtypes = []
         lib.sr_launch_count.restype = ctypes.c_int64
+        lib.sr_set_wait_limit.argtypes = [ctypes.c_int64]
+        lib.sr_set_wait_limit.restype = ctypes.c_int64
+        lib.sr_test_lose_arrival.argtypes = [i32]
         lib.sr_status_string.argtypes = [i32]
         lib.sr_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -183,3 +186,13 @@ def sr_device_status() -> int:
 def sr_launch_count() -> int:
     """Kernels launched by the library in this process so far."""
     return int(load_library().sr_launch_count())
+
+
+def sr_set_wait_limit(cycles: int) -> int:
+    """Cycle budget of the device-side waits of later launches; returns the previous budget."""
+    return int(load_library().sr_set_wait_limit(int(cycles)))
+
+
+def sr_test_lose_arrival(launches: int) -> None:
+    """Test hook: the next `launches` tensor-core regression launches leave out one barrier arrival."""
+    _check(load_library().sr_test_lose_arrival(int(launches)), "sr_test_lose_arrival")

@@ -27,6 +27,31 @@ int* device_status_word()
     return cache[dev];
 }
 
+static std::atomic<long long> g_wait_limit{1ll << 31};
+static std::atomic<int> g_lose_arrival{0};
+
+long long wait_cycle_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
+
+bool take_injected_lost_arrival()
+{
+    int n = g_lose_arrival.load(std::memory_order_relaxed);
+    while (n > 0 && !g_lose_arrival.compare_exchange_weak(n, n - 1, std::memory_order_relaxed)) {}
+    return n > 0;
+}
+
+int sm_count()
+{
+    static int cache[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (cache[dev] <= 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 1;
+        cache[dev] = n;
+    }
+    return cache[dev];
+}
+
 // Keys cubic-convolution weights (a = -0.75) for every phase of an integer scale, computed in
 // double and rounded once. src = (X + 1/2)/r - 1/2 = (2X + 1 - r) / (2r) in exact integers.
 // `bilinear`: the same four-tap window with weights (0, 1 - t, t, 0), so every kernel serves both forms.
@@ -183,6 +208,19 @@ const char* sr_status_string(int status)
 }
 
 int64_t sr_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+int64_t sr_set_wait_limit(int64_t cycles)
+{
+    if (cycles < 1) return (int64_t)g_wait_limit.load(std::memory_order_relaxed);
+    return (int64_t)g_wait_limit.exchange((long long)cycles, std::memory_order_relaxed);
+}
+
+int sr_test_lose_arrival(int launches)
+{
+    if (launches < 0) return SR_ERR_SHAPE;
+    g_lose_arrival.store(launches, std::memory_order_relaxed);
+    return SR_OK;
+}
 
 int sr_device_status(void* stream, int* out_status)
 {

@@ -119,7 +119,7 @@ static cudaError_t launch_block(const float* lr, float* hr, const Problem& pb, c
 {
     const int64_t total = (int64_t)pb.n * pb.c * ((pb.H + 3) >> 2) * ((pb.W + 3) >> 2);
     int64_t blocks = (total + 255) / 256;
-    const int64_t cap = 148 * 8 * 4;
+    const int64_t cap = (int64_t)sm_count() * 8 * 4;
     if (blocks > cap) blocks = cap;
     bicubic_block_kernel<R><<<(unsigned)blocks, 256, 0, st>>>(lr, hr, pb);
     count_launches(1);
@@ -133,7 +133,7 @@ cudaError_t launch_bicubic(const float* lr, float* hr, const Problem& pb, cudaSt
     if (pb.r == 1) return launch_block<1>(lr, hr, pb, st);
     const int64_t total = (int64_t)pb.n * pb.c * pb.H * ((pb.W + 3) >> 2);
     int64_t blocks = (total + 255) / 256;
-    const int64_t cap = 148 * 8 * 4;
+    const int64_t cap = (int64_t)sm_count() * 8 * 4;
     if (blocks > cap) blocks = cap;
     bicubic_kernel<<<(unsigned)blocks, 256, 0, st>>>(lr, hr, pb);
     count_launches(1);

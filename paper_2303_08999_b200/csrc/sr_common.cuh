@@ -42,6 +42,15 @@ BicubicPhases make_phases(int scale, bool bilinear);
 // Address of the per-device status word (device memory; 0 = ok). Returns nullptr on a CUDA error.
 int* device_status_word();
 
+// Cycle budget of one device-side wait for the launches that follow (set by sr_set_wait_limit).
+long long wait_cycle_limit();
+
+// Test hook (sr_test_lose_arrival): true once per armed launch; the launch then leaves out one barrier arrival.
+bool take_injected_lost_arrival();
+
+// Multiprocessors of the current device (queried once per device; at least 1).
+int sm_count();
+
 // Adds to the process-wide count of kernels launched (read back by sr_launch_count).
 void count_launches(int n);
 

@@ -49,45 +49,69 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
     return done != 0;
 }
 
-// Cycle budget of one wait (about a second at B200 clocks).
+// Default cycle budget of one wait (about a second at B200 clocks); the host can lower it per launch.
 constexpr long long kWaitCycleLimit = 1ll << 31;
+// Budget of the waits a CTA makes while it winds down after a failed wait (copies and MMAs still in flight finish
+// within microseconds; a phase that can never complete must not hold the exit up for long).
+constexpr long long kDrainCycleLimit = 1ll << 21;
+
+// Per-CTA state of the bounded waits (shared memory): the flag a thread raises when its wait ran out, which every
+// other wait of the CTA polls, and the cycle budget of one wait.
+struct WaitCtx {
+    int abort_flag;
+    int reserved;
+    long long limit;
+};
 
 // Whole-warp wait: lane 0 polls, the result is broadcast. Returns the same value in every lane.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag);
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc);
 
 // Waits for the phase with the given parity to complete. Returns false when the budget ran out or
-// another thread of the CTA has already raised `*abort_flag` (a shared-memory word).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
+// another thread of the CTA has already raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    const long long limit = const_cast<const WaitCtx*>(wc)->limit;   // fixed for the launch: read once, not per poll
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycleLimit) {
-            *abort_flag = 1;
+        if (wc->abort_flag) return false;
+        if (clock64() - t0 > limit) {
+            wc->abort_flag = 1;
             return false;
         }
     }
 }
 
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
+// A wait of the wind-down after a failure: own short budget, ignores (and never raises) the abort flag.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kDrainCycleLimit) return false;
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc)
 {
     int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, wc) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
-    // lanes other than 0 did not observe the barrier themselves: one successful test gives them the acquire
-    if (ok) while (!mbar_try_wait(bar, parity, 0u)) {}
-    return ok != 0;
+    // Lanes other than 0 did not observe the barrier themselves: one successful test gives them the acquire. The
+    // phase lane 0 saw complete cannot be left behind before this warp has used it, so that test succeeds; a lane
+    // whose test fails all the same falls back to the bounded wait, and the warp agrees on the outcome.
+    if (ok && !mbar_try_wait(bar, parity, 0u)) ok = mbar_wait(bar, parity, wc) ? 1 : 0;
+    return __all_sync(0xffffffffu, ok != 0);
 }
 
 // Whole-warp wait in which every lane tests the barrier itself (one shared-memory round trip when the phase is
 // already complete, against three for mbar_wait_warp: lane 0's test, the shuffle, the other lanes' test). `seen`:
 // the result of a test issued earlier (true = the phase was already complete then, nothing left to do).
-__device__ __forceinline__ bool mbar_wait_lanes(uint64_t* bar, uint32_t parity, volatile int* abort_flag, bool seen)
+__device__ __forceinline__ bool mbar_wait_lanes(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc, bool seen)
 {
     if (__all_sync(0xffffffffu, seen)) return true;
-    return mbar_wait(bar, parity, abort_flag);
+    return mbar_wait(bar, parity, wc);
 }
 
 // ---- proxies / fences ----------------------------------------------------------------------------------------------

@@ -101,3 +101,11 @@ def test_binding_refuses_cpu_tensors():
         sr.sr_bicubic_upsample(torch.zeros(1, 1, 2, 2), 2)
     with pytest.raises(TypeError):
         sr.sr_bilinear_upsample(torch.zeros(1, 1, 2, 2), 2)
+
+
+def test_wait_limit_is_returned_and_the_hook_validates_its_count(lib):
+    old = sr.sr_set_wait_limit(12345)
+    assert sr.sr_set_wait_limit(0) == 12345      # < 1: nothing changes, the current budget comes back
+    assert sr.sr_set_wait_limit(old) == 12345
+    assert lib.sr_test_lose_arrival(-1) == api.SR_ERR_SHAPE
+    assert lib.sr_test_lose_arrival(0) == api.SR_OK

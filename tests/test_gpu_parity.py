@@ -11,7 +11,7 @@ import torch
 import oracle
 import paper_2303_08999_b200 as sr
 import sr_inputs
-from gpu_util import TOL_F16, TOL_F32, dev, host, max_abs_err, tol_for
+from gpu_util import TOL_F16, TOL_F32, dev, host, max_abs_err, signed_asymmetric_dictionary, signed_gamma, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -209,3 +209,99 @@ def test_selected_with_ties(D, s, w):
     assert max_abs_err(got, want) <= TOL_F16
     got = host(sr.sr_dict_regress_selected(dev(lr), sel, idx, None, dev(dict_), 2, 5, s, sr.SR_COEF_COMPACT))
     assert max_abs_err(got, want) <= TOL_F16
+
+
+# ------------------------------------------------------------------ orientation and sign of the taps
+
+SIGNED_CASES = [
+    # n, c, h, w, r, D, k, dtype, s
+    (1, 3, 24, 64, 2, 72, 5, "f16", 8),    # every mode on the tensor-core kernel
+    (2, 3, 33, 50, 4, 72, 5, "f16", 8),    # HR width 200: dense / in-kernel selection / subset on the tensor cores, index planes on the general kernel
+    (1, 3, 20, 30, 2, 72, 5, "f32", 8),    # fp32 coefficients: general kernel
+    (1, 3, 12, 40, 2, 32, 7, "f16", 4),
+    (1, 3, 12, 32, 2, 72, 3, "f16", 12),
+    (1, 1, 9, 16, 2, 7, 9, "f32", 3),      # 9 x 9 atoms: general kernel
+    (1, 3, 30, 35, 4, 72, 5, "f16", 8),    # HR width 140: general kernel with binary16 coefficients
+    (1, 3, 40, 64, 4, 72, 5, "f16", 8),    # several 16-row tiles, two tile columns
+]
+
+
+@pytest.mark.parametrize("case", SIGNED_CASES, ids=lambda c: "-".join(map(str, c)))
+def test_signed_asymmetric_dictionary_and_negative_gamma_all_modes(case):
+    """Atoms without any symmetry and with both signs, re-weights with both signs: a 180-degree tap flip, a transposed
+    patch or a lost sign in the binary16 hi / lo split of the dictionary fails here (it passes with the generator's
+    point-symmetric, non-negative atoms)."""
+    n, c, h, w, r, D, k, dt, s = case
+    wl = _wl(n, c, h, w, r, D, k, dt)
+    lr, dict_, coef = sr_inputs.make_inputs(wl)
+    dict_ = signed_asymmetric_dictionary(dict_)
+    assert (dict_ < 0).any() and not np.allclose(dict_.reshape(D, k, k), dict_.reshape(D, k, k)[:, ::-1, ::-1])
+    tol = tol_for(coef)
+    dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
+    got = host(sr.sr_dict_regress_dense(dlr, dco, ddi, r, k))
+    assert max_abs_err(got, oracle.dict_regress_dense(lr, coef, dict_, r, k)) <= tol
+    want = oracle.dict_regress_selected(lr, coef, None, None, dict_, r, k, s)
+    got = host(sr.sr_dict_regress_selected(dlr, dco, None, None, ddi, r, k, s))
+    assert max_abs_err(got, want) <= tol
+    idx, sel = sr.sr_dict_select(dco, s, want_sel=True)
+    got = host(sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, r, k, s))
+    assert max_abs_err(got, want) <= tol
+    got = host(sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, r, k, s, sr.SR_COEF_COMPACT))
+    assert max_abs_err(got, want) <= tol
+    rng = np.random.default_rng(5)
+    S = rng.choice(D, size=s, replace=False).astype(np.uint8)
+    S[0] = 1 if 1 not in S[1:] else S[0]                     # the off-centre delta atom is in the subset
+    gamma = signed_gamma(s)
+    assert (gamma < 0).any()
+    want = oracle.dict_regress_selected(lr, coef, S, gamma, dict_, r, k, s, flags=oracle.IDX_GLOBAL)
+    got = host(sr.sr_dict_regress_selected(dlr, dco, dev(S), dev(gamma), ddi, r, k, s, sr.SR_IDX_GLOBAL))
+    assert max_abs_err(got, want) <= tol
+    compact = dev(coef[:, S.astype(int)].copy())
+    got = host(sr.sr_dict_regress_selected(dlr, compact, dev(S), dev(gamma), ddi, r, k, s, sr.SR_IDX_GLOBAL | sr.SR_COEF_COMPACT))
+    assert max_abs_err(got, want) <= tol
+    assert sr.sr_device_status() == 0
+
+
+@pytest.mark.parametrize("dt,w", [("f16", 48), ("f32", 48), ("f16", 35)])
+@pytest.mark.parametrize("tap", [(0, 1), (4, 0), (3, 4), (2, 2)])
+def test_off_centre_delta_atom_shifts_the_upsampled_image(dt, w, tap):
+    """One atom that is a single tap at (a, b), one-hot coefficients: the output is the up-sampled image read at
+    (Y + a - p, X + b - p), clamped to the frame. The expected frame is built from the bicubic oracle by indexing
+    alone, so the pairing of taps and patch positions is checked without the oracle's own regression."""
+    a, b = tap
+    r, k, D, p = 4, 5, 72, 2
+    wl = _wl(1, 3, 20, w, r, D, k, dt)
+    lr, dict_, _ = sr_inputs.make_inputs(wl)
+    dict_[3] = 0
+    dict_[3, a * k + b] = 1
+    coef = np.zeros((1, D, wl.H, wl.W), np.float16 if dt == "f16" else np.float32)
+    coef[:, 3] = 1
+    U = oracle.bicubic_upsample(lr, r)
+    yy = np.clip(np.arange(wl.H) + a - p, 0, wl.H - 1)
+    xx = np.clip(np.arange(wl.W) + b - p, 0, wl.W - 1)
+    want = U[:, :, yy][:, :, :, xx]
+    dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
+    assert max_abs_err(host(sr.sr_dict_regress_dense(dlr, dco, ddi, r, k)), want) <= 2e-6
+    assert max_abs_err(host(sr.sr_dict_regress_selected(dlr, dco, None, None, ddi, r, k, 3)), want) <= 2e-6
+    S = np.array([0, 3, 5], np.uint8)
+    assert max_abs_err(host(sr.sr_dict_regress_selected(dlr, dco, dev(S), None, ddi, r, k, 3, sr.SR_IDX_GLOBAL)), want) <= 2e-6
+    idx, sel = sr.sr_dict_select(dco, 3, want_sel=True)
+    assert max_abs_err(host(sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, r, k, 3, sr.SR_COEF_COMPACT)), want) <= 2e-6
+    np.testing.assert_allclose(oracle.dict_regress_dense(lr, coef, dict_, r, k), want, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("scale,bound", [(2.0 ** 15, TOL_F16 * 2.0 ** 15), (2.0 ** -10, 1e-5)])
+def test_dictionary_magnitude_range_of_the_tensor_core_path(scale, bound):
+    """The tensor-core path keeps the fp32 dictionary as a binary16 hi + lo pair, so its taps must stay below the
+    largest binary16 number (65504); taps below 2^-14 fall into the binary16 subnormals and keep an absolute, not a
+    relative, precision (2^-25 per tap). A large dictionary (taps up to about 9500) must be as accurate relative to
+    its scale as the ordinary one; a tiny one (taps around 1e-4) within the absolute bound that follows from 2^-25 per
+    tap: 3 (sum of |coefficients|) x 25 taps x 1.45 (|U|) x 2^-25 = 3.3e-6."""
+    wl = _wl(1, 3, 24, 64, 2, 72, 5, "f16")
+    lr, dict_, coef = sr_inputs.make_inputs(wl)
+    dict_ = (signed_asymmetric_dictionary(dict_) * np.float32(scale)).astype(np.float32)
+    assert np.abs(dict_).max() < 65504
+    got = host(sr.sr_dict_regress_dense(dev(lr), dev(coef), dev(dict_), 2, 5))
+    assert max_abs_err(got, oracle.dict_regress_dense(lr, coef, dict_, 2, 5)) <= bound
+    got = host(sr.sr_dict_regress_selected(dev(lr), dev(coef), None, None, dev(dict_), 2, 5, 8))
+    assert max_abs_err(got, oracle.dict_regress_selected(lr, coef, None, None, dict_, 2, 5, 8)) <= bound

@@ -11,7 +11,7 @@ import pytest
 import oracle
 import paper_2303_08999_b200 as sr
 import sr_inputs
-from gpu_util import TOL_F16, dev, host
+from gpu_util import TOL_F16, dev, host, signed_asymmetric_dictionary
 
 pytestmark = pytest.mark.gpu
 
@@ -39,6 +39,8 @@ def test_random_shapes_all_modes(seed):
         lr, dict_, coef = sr_inputs.make_inputs(wl, seed=1000 * seed + case)
         if rng.random() < 0.4:   # coarse grid: exact magnitude ties, +/- pairs and zeros are frequent
             coef = (np.round(coef.astype(np.float32) * 64) / 64).astype(coef.dtype)
+        if case % 2:             # every second case: atoms without symmetry and with both signs
+            dict_ = signed_asymmetric_dictionary(dict_, seed=case)
         tag = f"seed {seed} case {case}: {wl}"
         dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
         err = np.abs(host(sr.sr_bicubic_upsample(dlr, r)).astype(np.float64) - oracle.bicubic_upsample(lr, r)).max()
@@ -55,7 +57,7 @@ def test_random_shapes_all_modes(seed):
         err = np.abs(host(sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, r, k, s, sr.SR_COEF_COMPACT)) - want).max()
         assert err <= TOL_F16, tag
         S = rng.choice(D, size=s, replace=False).astype(np.uint8)
-        gamma = rng.uniform(0.5, 1.5, size=s).astype(np.float32)
+        gamma = (rng.uniform(0.5, 1.5, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
         want = oracle.dict_regress_selected(lr, coef, S, gamma, dict_, r, k, s, flags=oracle.IDX_GLOBAL)
         err = np.abs(host(sr.sr_dict_regress_selected(dlr, dco, dev(S), dev(gamma), ddi, r, k, s, sr.SR_IDX_GLOBAL)) - want).max()
         assert err <= TOL_F16, tag
@@ -95,6 +97,8 @@ def test_random_shapes_random_flags(seed):
             lr, dict_, coef = sr_inputs.make_inputs(wl, seed=3000 * seed + case)
         if rng.random() < 0.4:
             coef = (np.round(coef.astype(np.float32) * 64) / 64).astype(coef.dtype)
+        if case % 2:
+            dict_ = signed_asymmetric_dictionary(dict_, seed=case)
         fl = ofl = 0
         if rng.random() < 0.5:
             fl, ofl = fl | sr.SR_CLAMP01, ofl | oracle.CLAMP01
@@ -120,7 +124,7 @@ def test_random_shapes_random_flags(seed):
         check(sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, r, k, s, fl), want)
         check(sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, r, k, s, fl | sr.SR_COEF_COMPACT), want)
         S = rng.choice(D, size=s, replace=False).astype(np.uint8)
-        gamma = rng.uniform(0.5, 1.5, size=s).astype(np.float32)
+        gamma = (rng.uniform(0.5, 1.5, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
         want = oracle.dict_regress_selected(lr, coef, S, gamma, dict_, r, k, s, flags=ofl | oracle.IDX_GLOBAL)
         check(sr.sr_dict_regress_selected(dlr, dco, dev(S), dev(gamma), ddi, r, k, s, fl | sr.SR_IDX_GLOBAL), want)
         up = (sr.sr_bilinear_upsample if bilinear else sr.sr_bicubic_upsample)(dlr, r)

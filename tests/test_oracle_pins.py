@@ -353,3 +353,25 @@ def test_generator_distributions_and_dictionary():
     np.testing.assert_array_equal(coef, coef2)
     half = sr_inputs.make_coef(sr_inputs.Workload("t", 1, 3, 32, 32, 2, coef_dtype="f16"))
     np.testing.assert_array_equal(half, sr_inputs.round_f16(coef))
+
+
+def test_binary16_widening_every_bit_pattern():
+    """The oracle widens binary16 coefficients itself (sign, exponent, mantissa; subnormals, infinities, NaN). Every one
+    of the 65536 bit patterns is pinned against numpy's own float16 -> float64 conversion, through the two routes a
+    coefficient takes: the selected values (`sel` of the selection) and the regression (a 1 x 1 unit atom on a
+    constant unit image returns the coefficient itself)."""
+    bits = np.arange(65536, dtype=np.uint16)
+    coef = bits.view(np.float16).reshape(1, 1, 256, 256)
+    want = coef.astype(np.float64)
+    _, sel = oracle.dict_select(coef, 1, want_sel=True)
+    finite = np.isfinite(want)
+    np.testing.assert_array_equal(sel[finite], want[finite])
+    np.testing.assert_array_equal(np.isnan(sel), np.isnan(want))
+    np.testing.assert_array_equal(sel[np.isinf(want)], want[np.isinf(want)])
+    assert np.array_equal(np.signbit(sel[finite]), np.signbit(want[finite]))      # -0 keeps its sign
+    # subnormals and the largest finite value, by hand
+    for b, v in ((0x0001, 2.0 ** -24), (0x03FF, 1023 * 2.0 ** -24), (0x0400, 2.0 ** -14), (0x7BFF, 65504.0), (0xFBFF, -65504.0)):
+        assert sel.reshape(-1)[b] == v
+    lr = np.ones((1, 1, 256, 256), np.float32)
+    out = oracle.dict_regress_dense(lr, coef, np.ones((1, 1), np.float32), 1, 1)
+    np.testing.assert_array_equal(out[0][finite[0]], want[0][finite[0]])
