@@ -4,6 +4,8 @@
 #include <atomic>
 
 #include "sr_common.cuh"
+#include "sr_regress_subset.cuh"
+#include "sr_regress_tc.cuh"
 #include "sr_umma.cuh"
 
 namespace sr {
@@ -104,6 +106,12 @@ static Problem make_problem(const sr_dims* d, int s, uint32_t flags)
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
+// Which tensor-core layout takes a dense launch. The second layout (sr_regress_tc.cu: channel-split epilogue, two CTAs
+// per SM, several rows per pipeline step) wins where the coefficient stream is light and the epilogue sets the pace:
+// few atoms, or 7 x 7 atoms with up to 32 of them; the first layout (sr_umma.cu) streams many atoms faster. Measured
+// on the 1080p sweep points (dense, D = 16 / 32 / 72 / 128; k = 3 / 5 / 7).
+static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 || (pb.k == 7 && pb.D <= 32); }
+
 } // namespace sr
 
 using namespace sr;
@@ -142,7 +150,10 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
         return SR_ERR_ALIGN;
     const Problem pb = make_problem(d, d->D, flags);
     cudaError_t err;
-    if (umma_supported(kModeDense, coef, coef_dtype, pb))
+    const bool first_ok = umma_supported(kModeDense, coef, coef_dtype, pb);
+    if (regress_tc_supported(kModeDense, coef, coef_dtype, pb) && (dense_prefers_second_layout(pb) || !first_ok))
+        err = launch_regress_tc(kModeDense, lr, coef, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
+    else if (first_ok)
         err = launch_regress_umma(kModeDense, lr, coef, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
     else
         err = launch_regress_fma(kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
@@ -186,7 +197,11 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     else mode = idx ? kModeIdx : kModeFusedSelect;
     cudaError_t err;
     const bool idx_vec_ok = !idx || (flags & SR_IDX_GLOBAL) || ((reinterpret_cast<uintptr_t>(idx) & 15) == 0);   // 16-byte reads
-    if (idx_vec_ok && umma_supported(mode, coef_or_sel, coef_dtype, pb))
+    if (regress_subset_supported(mode, coef_or_sel, coef_dtype, out, pb))
+        err = launch_regress_subset(lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
+    else if (regress_tc_supported(mode, coef_or_sel, coef_dtype, pb))
+        err = launch_regress_tc(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
+    else if (idx_vec_ok && umma_supported(mode, coef_or_sel, coef_dtype, pb))
         err = launch_regress_umma(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
     else
         err = launch_regress_fma(mode, lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, pb, (cudaStream_t)stream);

@@ -83,6 +83,36 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
+// The same wait for roles that have time to spare: between tests the thread sleeps, so that its polling does not take
+// issue slots and shared-memory cycles from the warps that set the pace.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    const long long limit = const_cast<const WaitCtx*>(wc)->limit;
+    while (true) {
+        __nanosleep(64);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (wc->abort_flag) return false;
+        if (clock64() - t0 > limit) {
+            wc->abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+// Whole-warp wait in which only lane 0 polls (the other lanes block at the warp barrier and take no issue slots or
+// shared-memory cycles meanwhile). Lane 0's successful test is an acquire; the warp barrier orders it before what the
+// other lanes do next. `relaxed`: lane 0 sleeps between tests. Returns the same value in every lane.
+__device__ __forceinline__ bool mbar_wait_leader(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc, bool relaxed)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = (relaxed ? mbar_wait_relaxed(bar, parity, wc) : mbar_wait(bar, parity, wc)) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
+}
+
 // A wait of the wind-down after a failure: own short budget, ignores (and never raises) the abort flag.
 __device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity)
 {
@@ -112,6 +142,14 @@ __device__ __forceinline__ bool mbar_wait_lanes(uint64_t* bar, uint32_t parity, 
 {
     if (__all_sync(0xffffffffu, seen)) return true;
     return mbar_wait(bar, parity, wc);
+}
+
+// The same, with an outcome the whole warp agrees on (the vote is only taken when the early test had failed): for
+// callers whose next instruction is warp-collective.
+__device__ __forceinline__ bool mbar_wait_lanes_uniform(uint64_t* bar, uint32_t parity, volatile WaitCtx* wc, bool seen)
+{
+    if (__all_sync(0xffffffffu, seen)) return true;
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, wc));
 }
 
 // ---- proxies / fences ----------------------------------------------------------------------------------------------

@@ -24,17 +24,18 @@ def _calls():
     lr, dict_, coef = sr_inputs.make_inputs(wl)
     dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
     idx, sel = sr.sr_dict_select(dco, 8, want_sel=True)
-    S = dev(np.arange(0, 72, 9, dtype=np.uint8))
+    S = dev(np.arange(0, 72, 6, dtype=np.uint8))          # twelve atoms: more than the FMA-pipe subset kernel (no waits) takes
     return {
         "dense": lambda: sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5),
         "fused_select": lambda: sr.sr_dict_regress_selected(dlr, dco, None, None, ddi, 2, 5, 8),
         "index_planes": lambda: sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, 2, 5, 8),
         "compact": lambda: sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, 2, 5, 8, sr.SR_COEF_COMPACT),
-        "global_subset": lambda: sr.sr_dict_regress_selected(dlr, dco, S, None, ddi, 2, 5, 8, sr.SR_IDX_GLOBAL),
+        "global_subset": lambda: sr.sr_dict_regress_selected(dlr, dco, S, None, ddi, 2, 5, 12, sr.SR_IDX_GLOBAL),
+        "dense_few_atoms": lambda: sr.sr_dict_regress_dense(dlr, dco[:, :16].contiguous(), ddi[:16].contiguous(), 2, 5),
     }
 
 
-@pytest.mark.parametrize("mode", ["dense", "fused_select", "index_planes", "compact", "global_subset"])
+@pytest.mark.parametrize("mode", ["dense", "fused_select", "index_planes", "compact", "global_subset", "dense_few_atoms"])
 def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_clean(mode):
     call = _calls()[mode]
     before = call().clone()
