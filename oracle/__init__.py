@@ -42,6 +42,12 @@ def _load():
         L.sr_ref_dict_regress_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp] + [i32] * 8 + [u32, i32]
         L.sr_ref_regress_at.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp, i64, vp] + [i32] * 8 + [u32, i32]
         L.sr_ref_dict_select_at.argtypes = [vp, i32, vp, i64, vp] + [i32] * 6
+        f64 = ctypes.c_double
+        L.sr_ref_selection_gram.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp] + [i32] * 7 + [u32, i32]
+        L.sr_ref_lasso_cd.argtypes = [vp, vp, i32, vp, f64, f64, vp, f64, i32, vp]
+        L.sr_ref_selection_search.argtypes = [vp, vp, f64, i32, f64, f64, f64, f64, f64, f64, i32, i32, vp, vp, vp, vp, i32, vp]
+        for f in (L.sr_ref_selection_gram, L.sr_ref_lasso_cd, L.sr_ref_selection_search):
+            f.restype = i32
         L.sr_ref_max_threads.argtypes = []
         for f in (L.sr_ref_bicubic_upsample, L.sr_ref_bilinear_upsample, L.sr_ref_dict_regress_dense, L.sr_ref_dict_select,
                   L.sr_ref_dict_regress_selected, L.sr_ref_regress_at, L.sr_ref_dict_select_at, L.sr_ref_max_threads):
@@ -150,3 +156,49 @@ def dict_select_at(coef, samples, s: int, threads: int = 0) -> np.ndarray:
     _check(_load().sr_ref_dict_select_at(coef.ctypes.data, _dtype_code(coef), samples.ctypes.data, samples.size,
                                          out.ctypes.data, n, H, W, D, s, threads), "select_at")
     return out
+
+
+def selection_gram(lr, coef, dict_, target, samples, scale: int, k: int, flags: int = 0, threads: int = 0):
+    """Gram statistics of the selection problem (Section III-A) over sampled flat [n][H][W] pixel indices
+    (None = every pixel): returns (G [L][L], b [L], hh) in float64."""
+    lr, coef, dict_, target = _c(lr, np.float32), _c(coef), _c(dict_, np.float32), _c(target, np.float32)
+    n, c, h, w = lr.shape
+    L = dict_.shape[0]
+    assert dict_.shape == (L, k * k) and coef.shape == (n, L, h * scale, w * scale) and target.shape == (n, c, h * scale, w * scale)
+    samples = None if samples is None else _c(samples, np.int64)
+    G = np.empty((L, L), dtype=np.float64)
+    b = np.empty(L, dtype=np.float64)
+    hh = ctypes.c_double(0.0)
+    _check(_load().sr_ref_selection_gram(lr.ctypes.data, coef.ctypes.data, _dtype_code(coef), dict_.ctypes.data, target.ctypes.data,
+                                         None if samples is None else samples.ctypes.data, 0 if samples is None else samples.size,
+                                         G.ctypes.data, b.ctypes.data, ctypes.addressof(hh), n, c, h, w, scale, k, L, flags, threads),
+           "selection_gram")
+    return G, b, float(hh.value)
+
+
+def lasso_cd(G, b, nrows: float, lam: float, beta0=None, active=None, tol: float = 1e-12, max_sweeps: int = 10000):
+    """Eq. 7 for one lambda by cyclic coordinate descent on the Gram matrix: returns (beta, sweeps)."""
+    G, b = _c(G, np.float64), _c(b, np.float64)
+    L = b.size
+    beta = np.ones(L) if beta0 is None else np.array(beta0, dtype=np.float64)
+    act = np.ones(L, dtype=np.uint8) if active is None else _c(active, np.uint8)
+    sweeps = ctypes.c_int(0)
+    _check(_load().sr_ref_lasso_cd(G.ctypes.data, b.ctypes.data, L, act.ctypes.data, float(nrows), float(lam), beta.ctypes.data,
+                                   float(tol), int(max_sweeps), ctypes.addressof(sweeps)), "lasso_cd")
+    return beta, int(sweeps.value)
+
+
+def selection_search(G, b, hh: float, nrows: float, alpha: float, delta_alpha: float, eps: float, lambda0: float,
+                     tol: float = 1e-12, max_sweeps: int = 10000, max_bisect: int = 30, max_steps: int = 64):
+    """Algorithm 1 on the Gram statistics: returns (idx uint8 [count], gamma float64 [count], trace [steps][6])."""
+    G, b = _c(G, np.float64), _c(b, np.float64)
+    L = b.size
+    idx = np.zeros(L, dtype=np.uint8)
+    gamma = np.zeros(L, dtype=np.float64)
+    trace = np.zeros((max_steps, 6), dtype=np.float64)
+    count, steps = ctypes.c_int(0), ctypes.c_int(0)
+    _check(_load().sr_ref_selection_search(G.ctypes.data, b.ctypes.data, float(hh), L, float(nrows), float(alpha), float(delta_alpha),
+                                           float(eps), float(lambda0), float(tol), int(max_sweeps), int(max_bisect), idx.ctypes.data,
+                                           gamma.ctypes.data, ctypes.addressof(count), trace.ctypes.data, max_steps,
+                                           ctypes.addressof(steps)), "selection_search")
+    return idx[: count.value].copy(), gamma[: count.value].copy(), trace[: steps.value].copy()

@@ -23,7 +23,13 @@
  * prefix / permutation identities, and a brute-force sort for the selection;
  * for the bilinear variant of stage 1a a library bilinear resize, closed-form
  * weights, exact reproduction of affine images away from the border and the
- * delta-atom identity.  No function here is parity-unpinned.
+ * delta-atom identity.  The selection search of Section III-A (Gram statistics,
+ * LASSO by coordinate descent, Algorithm 1, least-squares re-fit) is pinned in
+ * tests/test_oracle_pins_selection.py: the Gram matrix against per-atom
+ * responses built from the pinned dense regression, the LASSO against a library
+ * solver and its optimality conditions, the re-fit against a library least-squares
+ * solve, and the search against its stopping rules on hand-built problems.
+ * No function here is parity-unpinned.
  */
 #include <algorithm>
 #include <cmath>
@@ -252,6 +258,140 @@ void upsample_all(const float* lr, const Dims& d, std::vector<double>& U, unsign
         }
 }
 
+
+/* ---- dictionary selection search (Section III-A) ------------------------------------------------------------------
+ *
+ * The paper keeps alpha * L of the L atoms: a selecting vector beta enters the filter as F_{W,beta} = Phi diag(beta) D
+ * (Eq. 5 / Eq. 6; the printed sums over i = 0..L are read as the sum over atoms), so the model output at HR pixel i,
+ * channel c is y[i,c] = sum_l beta_l z_l[i,c] with the per-atom response
+ *       z_l[i,c] = Phi_l[i] * (dict_l . B_{i,c}),
+ * and the loss against the ground-truth image h is (1/N) || h - Z beta ||^2, N = number of rows (sampled pixels times
+ * channels; the paper's N is its batch size: a constant factor on lambda).  Everything the search needs from the
+ * images is the Gram matrix G = Z^T Z, b = Z^T h and h^T h.
+ */
+void selection_rows(const Dims& d, const float* lr, const void* coef, int dtype, const float* dict, unsigned flags,
+                    int frame, int Y, int X, double* z /* [c][L] */)
+{
+    const int k = d.k, p = d.p(), kk = k * k;
+    const int64_t HW = (int64_t)d.H() * d.W();
+    for (int ch = 0; ch < d.c; ++ch) {
+        const float* plane = lr + ((int64_t)frame * d.c + ch) * d.h * d.w;
+        double B[81];
+        for (int a = 0; a < k; ++a)
+            for (int b = 0; b < k; ++b) {
+                const int yy = clampi(Y + a - p, 0, d.H() - 1), xx = clampi(X + b - p, 0, d.W() - 1);
+                B[a * k + b] = (flags & REF_UPSAMPLE_BILINEAR) ? bilinear_at(plane, d.h, d.w, d.r, yy, xx)
+                                                                : bicubic_at(plane, d.h, d.w, d.r, yy, xx);
+            }
+        for (int l = 0; l < d.L; ++l) {
+            double resp = 0.0;
+            for (int j = 0; j < kk; ++j) resp += (double)dict[(int64_t)l * kk + j] * B[j];
+            const double phi = coef_at(coef, dtype, ((int64_t)frame * d.L + l) * HW + (int64_t)Y * d.W() + X);
+            z[ch * d.L + l] = phi * resp;
+        }
+    }
+}
+
+/* loss (1/N) (h^T h - 2 b^T beta + beta^T G beta) over the active atoms, summed in index order */
+double selection_loss(const double* G, const double* b, double hh, int L, const uint8_t* active, const double* beta, double nrows)
+{
+    double quad = 0.0, lin = 0.0;
+    for (int l = 0; l < L; ++l) {
+        if (!active[l]) continue;
+        double row = 0.0;
+        for (int m = 0; m < L; ++m)
+            if (active[m]) row += G[(int64_t)l * L + m] * beta[m];
+        quad += beta[l] * row;
+        lin += b[l] * beta[l];
+    }
+    return (hh - 2.0 * lin + quad) / nrows;
+}
+
+/*
+ * Eq. 7: beta = argmin (1/N) || h - Z beta ||^2 + lambda |beta|_1 over the active atoms, by cyclic coordinate descent
+ * on the Gram matrix.  r = b - G beta is kept up to date; one coordinate step is
+ *       rho = r_l + G_ll beta_l,   beta_l <- soft(rho, lambda N / 2) / G_ll,   r <- r - (beta_l_new - beta_l_old) G[:, l].
+ * Sweeps repeat until no coefficient moved by more than tol (or max_sweeps).  Returns the number of sweeps.
+ */
+int lasso_cd(const double* G, const double* b, int L, const uint8_t* active, double nrows, double lambda, double* beta,
+             double tol, int max_sweeps)
+{
+    std::vector<double> r(L, 0.0);
+    for (int l = 0; l < L; ++l) {
+        if (!active[l]) { beta[l] = 0.0; continue; }
+        double acc = 0.0;
+        for (int m = 0; m < L; ++m)
+            if (active[m]) acc += G[(int64_t)l * L + m] * beta[m];
+        r[l] = b[l] - acc;
+    }
+    const double thr = 0.5 * lambda * nrows;
+    int sweep = 0;
+    for (; sweep < max_sweeps; ++sweep) {
+        double moved = 0.0;
+        for (int l = 0; l < L; ++l) {
+            if (!active[l]) continue;
+            const double gll = G[(int64_t)l * L + l];
+            if (!(gll > 0.0)) continue;
+            const double rho = r[l] + gll * beta[l];
+            double nb = 0.0;
+            if (rho > thr) nb = (rho - thr) / gll;
+            else if (rho < -thr) nb = (rho + thr) / gll;
+            const double delta = nb - beta[l];
+            if (delta != 0.0) {
+                for (int m = 0; m < L; ++m)
+                    if (active[m]) r[m] -= delta * G[(int64_t)m * L + l];
+                beta[l] = nb;
+                if (std::fabs(delta) > moved) moved = std::fabs(delta);
+            }
+        }
+        if (moved <= tol) { ++sweep; break; }
+    }
+    return sweep;
+}
+
+int count_nonzero(const double* beta, int L, const uint8_t* active)
+{
+    int n = 0;
+    for (int l = 0; l < L; ++l) n += (active[l] && beta[l] != 0.0) ? 1 : 0;
+    return n;
+}
+
+/* Eq. 9: gamma = argmin || h - sum_{l in S} gamma_l z_l ||^2, i.e. G_SS gamma = b_S, by Cholesky (G_SS = R^T R).
+ * Returns false when G_SS is not positive definite. */
+bool refit_gamma(const double* G, const double* b, int L, const std::vector<int>& S, std::vector<double>& gamma)
+{
+    const int s = (int)S.size();
+    std::vector<double> A((size_t)s * s), y(s);
+    for (int i = 0; i < s; ++i) {
+        for (int j = 0; j < s; ++j) A[(size_t)i * s + j] = G[(int64_t)S[i] * L + S[j]];
+        y[i] = b[S[i]];
+    }
+    for (int j = 0; j < s; ++j) {                 /* lower-triangular factor in place, column by column */
+        double dj = A[(size_t)j * s + j];
+        for (int q = 0; q < j; ++q) dj -= A[(size_t)j * s + q] * A[(size_t)j * s + q];
+        if (!(dj > 0.0)) return false;
+        dj = std::sqrt(dj);
+        A[(size_t)j * s + j] = dj;
+        for (int i = j + 1; i < s; ++i) {
+            double v = A[(size_t)i * s + j];
+            for (int q = 0; q < j; ++q) v -= A[(size_t)i * s + q] * A[(size_t)j * s + q];
+            A[(size_t)i * s + j] = v / dj;
+        }
+    }
+    for (int i = 0; i < s; ++i) {                 /* forward, then backward substitution */
+        double v = y[i];
+        for (int q = 0; q < i; ++q) v -= A[(size_t)i * s + q] * y[q];
+        y[i] = v / A[(size_t)i * s + i];
+    }
+    for (int i = s - 1; i >= 0; --i) {
+        double v = y[i];
+        for (int q = i + 1; q < s; ++q) v -= A[(size_t)q * s + i] * y[q];
+        y[i] = v / A[(size_t)i * s + i];
+    }
+    gamma.assign(y.begin(), y.end());
+    return true;
+}
+
 } // namespace
 
 extern "C" {
@@ -436,6 +576,169 @@ int sr_ref_dict_select_at(const void* coef, int coef_dtype, const int64_t* sampl
         const int64_t f = samples[i] / HW, pix = samples[i] % HW;
         select_pixel(coef, coef_dtype, f * L * HW + pix, HW, L, s, idx_out + i * s);
     }
+    return REF_OK;
+}
+
+/*
+ * Gram statistics of the selection problem over sampled HR pixels (flat [n][H][W] indices; samples == NULL: every
+ * pixel), all channels of each: G [L][L] = Z^T Z, b [L] = Z^T h, *hh = h^T h, with the target image h [n][c][H][W].
+ */
+int sr_ref_selection_gram(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                          const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, int n, int c, int h,
+                          int w, int r, int k, int L, unsigned flags, int threads)
+{
+    if (!lr || !coef || !dict || !target || !G || !b || !hh) return REF_ERR_NULL;
+    const Dims d{n, c, h, w, r, k, L};
+    if (int e = check_dims(d)) return e;
+    if (c > 16) return REF_ERR_UNSUPPORTED;
+    const int64_t HW = (int64_t)d.H() * d.W();
+    const int64_t count = samples ? nsamples : (int64_t)n * HW;
+#ifdef _OPENMP
+    const int nt = threads > 0 ? threads : omp_get_max_threads();
+#else
+    const int nt = 1;
+#endif
+    std::vector<std::vector<double>> part(nt, std::vector<double>((size_t)L * L + L + 1, 0.0));
+    int bad = 0;
+#pragma omp parallel num_threads(nt)
+    {
+#ifdef _OPENMP
+        std::vector<double>& acc = part[omp_get_thread_num()];
+#else
+        std::vector<double>& acc = part[0];
+#endif
+        std::vector<double> z((size_t)c * L);
+#pragma omp for schedule(static)
+        for (int64_t si = 0; si < count; ++si) {
+            const int64_t flat = samples ? samples[si] : si;
+            if (flat < 0 || flat >= (int64_t)n * HW) { bad = 1; continue; }
+            const int frame = (int)(flat / HW);
+            const int64_t pix = flat % HW;
+            const int Y = (int)(pix / d.W()), X = (int)(pix % d.W());
+            selection_rows(d, lr, coef, coef_dtype, dict, flags, frame, Y, X, z.data());
+            for (int ch = 0; ch < c; ++ch) {
+                const double hv = (double)target[((int64_t)frame * c + ch) * HW + pix];
+                const double* zr = z.data() + (size_t)ch * L;
+                for (int l = 0; l < L; ++l) {
+                    for (int m = 0; m < L; ++m) acc[(size_t)l * L + m] += zr[l] * zr[m];
+                    acc[(size_t)L * L + l] += zr[l] * hv;
+                }
+                acc[(size_t)L * L + L] += hv * hv;
+            }
+        }
+    }
+    if (bad) return REF_ERR_SHAPE;
+    for (int64_t i = 0; i < (int64_t)L * L; ++i) { double v = 0.0; for (int t = 0; t < nt; ++t) v += part[t][i]; G[i] = v; }
+    for (int l = 0; l < L; ++l) { double v = 0.0; for (int t = 0; t < nt; ++t) v += part[t][(size_t)L * L + l]; b[l] = v; }
+    { double v = 0.0; for (int t = 0; t < nt; ++t) v += part[t][(size_t)L * L + L]; *hh = v; }
+    return REF_OK;
+}
+
+/* Eq. 7 for one lambda; beta holds the start on entry and the solution on return; *sweeps the sweeps used. */
+int sr_ref_lasso_cd(const double* G, const double* b, int L, const uint8_t* active, double nrows, double lambda,
+                    double* beta, double tol, int max_sweeps, int* sweeps)
+{
+    if (!G || !b || !active || !beta) return REF_ERR_NULL;
+    if (L < 1 || L > 256 || !(nrows > 0.0) || !(lambda >= 0.0)) return REF_ERR_SHAPE;
+    const int n = lasso_cd(G, b, L, active, nrows, lambda, beta, tol, max_sweeps);
+    if (sweeps) *sweeps = n;
+    return REF_OK;
+}
+
+/*
+ * Algorithm 1 on the Gram statistics.  Step t lowers the kept fraction to alpha_{t+1} = max(alpha, alpha_t -
+ * delta_alpha) and looks for a lambda whose LASSO solution keeps alpha_{t+1} L atoms within eps L:
+ *   - lambda starts from the previous step's value and is doubled until || beta ||_0 <= alpha_{t+1} L;
+ *   - then lambda is bisected between the last two values of the doubling.  (The printed listing brackets
+ *     [lambda, 2 lambda] after its last doubling and moves the left end when too few atoms survive, which cannot
+ *     approach the target; it is read as the bracket of the last doubling step, as the text says, with the ends
+ *     moved the way a bisection needs: too few atoms -> lower the right end, too many -> raise the left end.)
+ *     If no lambda lands inside the band within max_bisect halvings, the feasible solution with the most atoms is kept;
+ *   - the weights of the coefficient layer are re-fitted on the kept atoms by least squares (Eq. 9): gamma solves
+ *     G_SS gamma = b_S; the re-fit layer replaces the old one, i.e. G <- diag(gamma) G_SS diag(gamma), b <- gamma b_S,
+ *     and beta restarts from 1 on the kept atoms.
+ * Output: the kept atoms in ascending order, the product of their re-weights over all steps, and per step
+ * trace[t][0..5] = alpha_{t+1}, lambda used, atoms kept, loss after the beta step, loss after the re-fit, LASSO solves.
+ */
+int sr_ref_selection_search(const double* G_in, const double* b_in, double hh, int L, double nrows, double alpha,
+                            double delta_alpha, double eps, double lambda0, double tol, int max_sweeps, int max_bisect,
+                            uint8_t* idx_out, double* gamma_out, int* count_out, double* trace, int max_steps, int* steps_out)
+{
+    if (!G_in || !b_in || !idx_out || !gamma_out || !count_out) return REF_ERR_NULL;
+    if (L < 1 || L > 256 || !(nrows > 0.0) || !(alpha > 0.0) || !(alpha <= 1.0) || !(delta_alpha > 0.0) || !(lambda0 > 0.0) || !(eps >= 0.0))
+        return REF_ERR_SHAPE;
+    std::vector<double> G(G_in, G_in + (size_t)L * L), b(b_in, b_in + L), beta(L, 1.0), gtot(L, 1.0), best(L), cand(L);
+    std::vector<uint8_t> active(L, 1);
+    double alpha_t = 1.0, lambda = lambda0;
+    int step = 0;
+    while (alpha_t > alpha + 1e-12 && step < max_steps) {        /* until alpha_t <= alpha (up to rounding of the schedule) */
+        const double alpha_next = std::max(alpha, 1.0 - (double)(step + 1) * delta_alpha);   /* alpha_t - delta_alpha, without the rounding of repeated subtraction */
+        const double target = alpha_next * L, band = eps * L;
+        int solves = 0;
+        int nnz = count_nonzero(beta.data(), L, active.data());
+        double lam_used = lambda, lam_hi = lambda;
+        bool have = false;                                   /* `best` holds a feasible solution (nnz <= target) */
+        int best_nnz = -1;
+        double best_lam = lambda;
+        /* doubling */
+        while ((double)nnz > target) {
+            cand = beta;
+            lasso_cd(G.data(), b.data(), L, active.data(), nrows, lambda, cand.data(), tol, max_sweeps);
+            ++solves;
+            nnz = count_nonzero(cand.data(), L, active.data());
+            beta = cand;
+            lam_hi = lambda;
+            lambda = 2.0 * lambda;
+        }
+        best = beta; best_nnz = nnz; best_lam = lam_hi; have = true;
+        /* bisection inside the last doubling step */
+        double left = 0.5 * lam_hi, right = lam_hi;
+        int it = 0;
+        while (std::fabs(target - (double)nnz) > band && it < max_bisect) {
+            const double mid = 0.5 * (left + right);
+            cand = best;
+            lasso_cd(G.data(), b.data(), L, active.data(), nrows, mid, cand.data(), tol, max_sweeps);
+            ++solves;
+            ++it;
+            nnz = count_nonzero(cand.data(), L, active.data());
+            if ((double)nnz <= target && nnz > best_nnz) { best = cand; best_nnz = nnz; best_lam = mid; }
+            if ((double)nnz < target) right = mid;
+            else if ((double)nnz > target) left = mid;
+            if (std::fabs(target - (double)nnz) <= band && (double)nnz <= target) { best = cand; best_nnz = nnz; best_lam = mid; }
+        }
+        (void)have;
+        beta = best;
+        lam_used = best_lam;
+        lambda = best_lam;
+        const double loss_beta = selection_loss(G.data(), b.data(), hh, L, active.data(), beta.data(), nrows);
+        /* W-step: re-fit on the support */
+        std::vector<int> S;
+        for (int l = 0; l < L; ++l)
+            if (active[l] && beta[l] != 0.0) S.push_back(l);
+        if (S.empty()) return REF_ERR_UNSUPPORTED;
+        std::vector<double> gamma;
+        if (!refit_gamma(G.data(), b.data(), L, S, gamma)) return REF_ERR_UNSUPPORTED;
+        std::fill(active.begin(), active.end(), (uint8_t)0);
+        for (size_t i = 0; i < S.size(); ++i) active[S[i]] = 1;
+        for (size_t i = 0; i < S.size(); ++i) {
+            for (size_t j = 0; j < S.size(); ++j) G[(size_t)S[i] * L + S[j]] = gamma[i] * G[(size_t)S[i] * L + S[j]] * gamma[j];
+            b[S[i]] = gamma[i] * b[S[i]];
+            gtot[S[i]] = gtot[S[i]] * gamma[i];
+        }
+        for (int l = 0; l < L; ++l) beta[l] = active[l] ? 1.0 : 0.0;
+        const double loss_gamma = selection_loss(G.data(), b.data(), hh, L, active.data(), beta.data(), nrows);
+        if (trace) {
+            double* tr = trace + (size_t)step * 6;
+            tr[0] = alpha_next; tr[1] = lam_used; tr[2] = (double)S.size(); tr[3] = loss_beta; tr[4] = loss_gamma; tr[5] = (double)solves;
+        }
+        alpha_t = alpha_next;
+        ++step;
+    }
+    int cnt = 0;
+    for (int l = 0; l < L; ++l)
+        if (active[l]) { idx_out[cnt] = (uint8_t)l; gamma_out[cnt] = gtot[l]; ++cnt; }
+    *count_out = cnt;
+    if (steps_out) *steps_out = step;
     return REF_OK;
 }
 
