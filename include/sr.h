@@ -50,6 +50,7 @@
 #ifndef SR_H_
 #define SR_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -142,6 +143,56 @@ int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, co
 int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_dtype, const uint8_t* idx,
                              const float* gamma, const float* dict, float* out, const sr_dims* d, int s,
                              uint32_t flags, void* stream);
+
+/*
+ * Dictionary selection search (Section III-A).  The paper keeps alpha * L of the L atoms: a selecting vector beta
+ * enters the filter as F = Phi diag(beta) D (Eq. 5-6), beta is found by LASSO (Eq. 7) with lambda doubled and then
+ * bisected until about alpha_t L atoms survive, the coefficient layer is re-fitted on the survivors by least squares
+ * (Eq. 9: one re-weight gamma_l per kept atom), and alpha_t is lowered step by step (Algorithm 1).  Fine-tuning the
+ * whole network is not part of this library; the re-fit of Eq. 9 is the paper's own fast substitute for it.  The
+ * result (atom ids + re-weights) is what sr_dict_regress_selected takes with SR_IDX_GLOBAL.
+ *
+ * sr_selection_gram: everything the search needs from the images.  With z_l[i,c] = coef[l][i] * (dict[l] . B_{i,c})
+ * the response of atom l alone at HR pixel i, channel c, and `target` [n][c][H][W] fp32 the ground-truth HR image:
+ *     G[l][m] = sum z_l z_m,   b[l] = sum z_l target,   *hh = sum target^2      (device fp64: G [D][D], b [D], hh [1])
+ * summed over the pixels listed in `samples` (device int64 flat [n][H][W] indices, nsamples of them; the paper samples
+ * its LASSO features too) or over every pixel when samples == NULL, all c channels of each.  Indices outside the
+ * tensor are skipped.  flags: SR_UPSAMPLE_BILINEAR or 0.  fp32 arithmetic per 32 pixels, fp64 accumulation; the result
+ * does not depend on the order in which thread blocks run.
+ * `scratch` is device memory of at least sr_selection_gram_scratch_bytes(d) bytes, 8-byte aligned; the call
+ * overwrites it, and two calls that share it must not overlap.  Returns SR_ERR_SHAPE when it is too small.
+ */
+size_t sr_selection_gram_scratch_bytes(const sr_dims* d);
+int sr_selection_gram(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                      const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const sr_dims* d,
+                      uint32_t flags, void* scratch, size_t scratch_bytes, void* stream);
+
+typedef struct sr_search_opts {
+    double alpha;        /* fraction of the atoms to keep in the end, in (0, 1]                                   */
+    double delta_alpha;  /* the kept fraction falls by this much per step (alpha_{t+1} = alpha_t - delta_alpha)    */
+    double eps;          /* a step accepts || beta ||_0 within eps * D of alpha_t * D                              */
+    double lambda0;      /* the small lambda the first step starts from (> 0)                                      */
+    double tol;          /* coordinate descent stops when no coefficient moved by more than tol in a sweep         */
+    int32_t max_sweeps;  /* ... or after this many sweeps                                                          */
+    int32_t max_bisect;  /* halvings of the lambda bracket per step                                                */
+    int32_t max_steps;   /* rows of `trace`; the search stops after this many steps                                */
+} sr_search_opts;
+
+/*
+ * sr_selection_search: Algorithm 1 on the Gram statistics (device pointers G [D][D], b [D], hh [1] in fp64, as
+ * sr_selection_gram writes them; nrows = number of (pixel, channel) rows they were summed over: the 1/N of Eq. 7),
+ * D <= 128.  Writes, all on the device: idx_out [D] the kept atoms in ascending order, gamma_out [D] their re-weights
+ * (product over all steps), *count_out how many were kept (-1 when a re-fit met a singular matrix), and per step
+ * trace[t][0..5] = alpha_t, lambda used, atoms kept, loss after the beta step, loss after the re-fit, LASSO solves
+ * (trace and steps_out may be NULL).  The printed listing's bisection is read as a bisection inside the last doubling
+ * step with the feasible solution that keeps the most atoms taken when no lambda lands in the band.
+ * `scratch`: device memory of at least sr_selection_search_scratch_bytes(D) bytes, 8-byte aligned.  fp64 throughout;
+ * one warp, every sum in a fixed order: the same inputs give the same bits on every run.
+ */
+size_t sr_selection_search_scratch_bytes(int32_t D);
+int sr_selection_search(const double* G, const double* b, const double* hh, double nrows, int32_t D,
+                        const sr_search_opts* opts, uint8_t* idx_out, float* gamma_out, int32_t* count_out, double* trace,
+                        int32_t* steps_out, void* scratch, size_t scratch_bytes, void* stream);
 
 /* Text for a status code (static storage, never NULL). */
 const char* sr_status_string(int status);

@@ -20,11 +20,17 @@ SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16 = 1
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
-           "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival")
+           "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival",
+           "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes")
 
 
 class sr_dims(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int32) for name in ("n", "c", "h", "w", "scale", "k", "D")]
+
+
+class sr_search_opts(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_double), ("delta_alpha", ctypes.c_double), ("eps", ctypes.c_double), ("lambda0", ctypes.c_double),
+                ("tol", ctypes.c_double), ("max_sweeps", ctypes.c_int32), ("max_bisect", ctypes.c_int32), ("max_steps", ctypes.c_int32)]
 
 
 class SrError(RuntimeError):
@@ -58,6 +64,13 @@ def load_library() -> ctypes.CDLL:
         lib.sr_set_wait_limit.argtypes = [ctypes.c_int64]
         lib.sr_set_wait_limit.restype = ctypes.c_int64
         lib.sr_test_lose_arrival.argtypes = [i32]
+        i64, f64, sz = ctypes.c_int64, ctypes.c_double, ctypes.c_size_t
+        lib.sr_selection_gram_scratch_bytes.argtypes = [dp]
+        lib.sr_selection_gram_scratch_bytes.restype = sz
+        lib.sr_selection_gram.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, dp, u32, vp, sz, vp]
+        lib.sr_selection_search_scratch_bytes.argtypes = [ctypes.c_int32]
+        lib.sr_selection_search_scratch_bytes.restype = sz
+        lib.sr_selection_search.argtypes = [vp, vp, vp, f64, ctypes.c_int32, ctypes.POINTER(sr_search_opts), vp, vp, vp, vp, vp, vp, sz, vp]
         lib.sr_status_string.argtypes = [i32]
         lib.sr_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -196,3 +209,55 @@ def sr_set_wait_limit(cycles: int) -> int:
 def sr_test_lose_arrival(launches: int) -> None:
     """Test hook: the next `launches` tensor-core regression launches leave out one barrier arrival."""
     _check(load_library().sr_test_lose_arrival(int(launches)), "sr_test_lose_arrival")
+
+
+def sr_selection_gram(lr, coef, dict_, target, samples, scale: int, k: int, flags: int = 0):
+    """Gram statistics of the dictionary selection search: returns (G [D][D], b [D], hh [1]) as float64 CUDA tensors.
+    `samples`: int64 CUDA tensor of flat [n][H][W] pixel indices, or None for every pixel."""
+    lr, dict_, target = _dev(lr, torch.float32, "lr"), _dev(dict_, torch.float32, "dict"), _dev(target, torch.float32, "target")
+    code = _coef_code(coef)
+    _dev(coef, coef.dtype, "coef")
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    assert dict_.shape == (D, k * k) and coef.shape == (n, D, h * scale, w * scale) and target.shape == (n, c, h * scale, w * scale)
+    if samples is not None:
+        _dev(samples, torch.int64, "samples")
+    d = sr_dims(n, c, h, w, scale, k, D)
+    lib = load_library()
+    nbytes = int(lib.sr_selection_gram_scratch_bytes(ctypes.byref(d)))
+    if nbytes == 0:
+        raise SrError(SR_ERR_UNSUPPORTED, "sr_selection_gram_scratch_bytes")
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=lr.device)
+    G = torch.empty((D, D), dtype=torch.float64, device=lr.device)
+    b = torch.empty(D, dtype=torch.float64, device=lr.device)
+    hh = torch.empty(1, dtype=torch.float64, device=lr.device)
+    _check(lib.sr_selection_gram(_ptr(lr), _ptr(coef), code, _ptr(dict_), _ptr(target), _ptr(samples),
+                                 0 if samples is None else samples.numel(), _ptr(G), _ptr(b), _ptr(hh), ctypes.byref(d), flags,
+                                 _ptr(scratch), nbytes, _stream()), "sr_selection_gram")
+    return G, b, hh
+
+
+def sr_selection_search(G, b, hh, nrows: float, alpha: float, delta_alpha: float, eps: float, lambda0: float, tol: float = 1e-9,
+                        max_sweeps: int = 2000, max_bisect: int = 30, max_steps: int = 64):
+    """Algorithm 1 on the Gram statistics (float64 CUDA tensors). Returns (idx uint8 [count], gamma float32 [count],
+    trace float64 [steps][6]) as CUDA tensors; reading the count synchronises the stream."""
+    _dev(G, torch.float64, "G"), _dev(b, torch.float64, "b"), _dev(hh, torch.float64, "hh")
+    D = b.numel()
+    assert G.shape == (D, D) and hh.numel() == 1
+    lib = load_library()
+    nbytes = int(lib.sr_selection_search_scratch_bytes(D))
+    if nbytes == 0:
+        raise SrError(SR_ERR_UNSUPPORTED, "sr_selection_search_scratch_bytes")
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=G.device)
+    idx = torch.zeros(D, dtype=torch.uint8, device=G.device)
+    gamma = torch.zeros(D, dtype=torch.float32, device=G.device)
+    count = torch.zeros(1, dtype=torch.int32, device=G.device)
+    steps = torch.zeros(1, dtype=torch.int32, device=G.device)
+    trace = torch.zeros((max_steps, 6), dtype=torch.float64, device=G.device)
+    o = sr_search_opts(alpha, delta_alpha, eps, lambda0, tol, max_sweeps, max_bisect, max_steps)
+    _check(lib.sr_selection_search(_ptr(G), _ptr(b), _ptr(hh), float(nrows), D, ctypes.byref(o), _ptr(idx), _ptr(gamma), _ptr(count),
+                                   _ptr(trace), _ptr(steps), _ptr(scratch), nbytes, _stream()), "sr_selection_search")
+    n = int(count.item())
+    if n < 0:
+        raise SrError(SR_ERR_UNSUPPORTED, "sr_selection_search: a re-fit met a singular matrix")
+    return idx[:n], gamma[:n], trace[: int(steps.item())]

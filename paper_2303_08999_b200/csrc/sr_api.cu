@@ -6,6 +6,7 @@
 #include "sr_common.cuh"
 #include "sr_regress_subset.cuh"
 #include "sr_regress_tc.cuh"
+#include "sr_selection.cuh"
 #include "sr_umma.cuh"
 
 namespace sr {
@@ -206,6 +207,54 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     else
         err = launch_regress_fma(mode, lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, pb, (cudaStream_t)stream);
     return err == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+size_t sr_selection_gram_scratch_bytes(const sr_dims* d)
+{
+    if (!d || d->D < 1 || d->D > 128) return 0;
+    return (size_t)selection_gram_slots() * selection_gram_slot_bytes(d->D);
+}
+
+int sr_selection_gram(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                      const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const sr_dims* d,
+                      uint32_t flags, void* scratch, size_t scratch_bytes, void* stream)
+{
+    if (!lr || !coef || !dict || !target || !G || !b || !hh || !d || !scratch) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (d->D > 128 || d->c > 16) return SR_ERR_UNSUPPORTED;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)SR_UPSAMPLE_BILINEAR) return SR_ERR_UNSUPPORTED;
+    if (samples && nsamples < 1) return SR_ERR_SHAPE;
+    if (!aligned(lr, 4) || !aligned(dict, 4) || !aligned(target, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4) ||
+        !aligned(G, 8) || !aligned(b, 8) || !aligned(hh, 8) || !aligned(scratch, 8) || (samples && !aligned(samples, 8)))
+        return SR_ERR_ALIGN;
+    const size_t slot = selection_gram_slot_bytes(d->D);
+    int nslots = selection_gram_slots();
+    if (scratch_bytes < slot) return SR_ERR_SHAPE;
+    if (scratch_bytes / slot < (size_t)nslots) nslots = (int)(scratch_bytes / slot);
+    const Problem pb = make_problem(d, d->D, flags);
+    return launch_selection_gram(lr, coef, coef_dtype, dict, target, samples, nsamples, G, b, hh, pb, static_cast<double*>(scratch),
+                                 nslots, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+size_t sr_selection_search_scratch_bytes(int32_t D) { return (D < 1 || D > 128) ? 0 : selection_search_scratch_bytes(D); }
+
+int sr_selection_search(const double* G, const double* b, const double* hh, double nrows, int32_t D,
+                        const sr_search_opts* o, uint8_t* idx_out, float* gamma_out, int32_t* count_out, double* trace,
+                        int32_t* steps_out, void* scratch, size_t scratch_bytes, void* stream)
+{
+    if (!G || !b || !hh || !o || !idx_out || !gamma_out || !count_out || !scratch) return SR_ERR_NULL;
+    if (D < 1 || !(nrows > 0.0)) return SR_ERR_SHAPE;
+    if (D > 128) return SR_ERR_UNSUPPORTED;
+    if (!(o->alpha > 0.0) || !(o->alpha <= 1.0) || !(o->delta_alpha > 0.0) || !(o->lambda0 > 0.0) || !(o->eps >= 0.0) ||
+        !(o->tol >= 0.0) || o->max_sweeps < 1 || o->max_bisect < 0 || o->max_steps < 1)
+        return SR_ERR_SHAPE;
+    if (!aligned(G, 8) || !aligned(b, 8) || !aligned(hh, 8) || !aligned(scratch, 8) || !aligned(gamma_out, 4) ||
+        !aligned(count_out, 4) || (trace && !aligned(trace, 8)) || (steps_out && !aligned(steps_out, 4)))
+        return SR_ERR_ALIGN;
+    if (scratch_bytes < selection_search_scratch_bytes(D)) return SR_ERR_SHAPE;
+    return launch_selection_search(G, b, hh, nrows, D, *o, idx_out, gamma_out, count_out, trace, steps_out,
+                                   static_cast<double*>(scratch), (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
 }
 
 const char* sr_status_string(int status)
