@@ -83,7 +83,8 @@ enum {
     SR_ERR_UNSUPPORTED = 3, /* scale not in [1,8]; k even or > 9; D > 256; unknown dtype or flag */
     SR_ERR_ALIGN = 4,       /* a pointer is not aligned to its element size      */
     SR_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed              */
-    SR_ERR_TIMEOUT = 6      /* device status only: a bounded device-side wait expired */
+    SR_ERR_TIMEOUT = 6,     /* device status only: a bounded device-side wait expired */
+    SR_ERR_TOO_LARGE = 7    /* sr_selection_gram_static: more atoms than its built-in scratch holds */
 };
 
 /*
@@ -166,6 +167,25 @@ size_t sr_selection_gram_scratch_bytes(const sr_dims* d);
 int sr_selection_gram(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
                       const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const sr_dims* d,
                       uint32_t flags, void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * sr_selection_gram for callers that cannot allocate device memory where they need the statistics: a pipeline that
+ * sizes every buffer once at start-up and then runs under a fixed memory budget, a plug-in whose host application owns
+ * the allocator, a service that keeps cudaMalloc (which synchronises the whole device and can fail late) out of its
+ * steady state.  Same inputs, outputs and results as sr_selection_gram, but no `scratch` argument: the per-block fp64
+ * partial sums live in a device array that is part of the library, 1 660 928 bytes (32 blocks x (80 x 80 + 80 + 8)
+ * doubles) held by every GPU that loads the library until the process exits.  Limit: d->D <= 80 atoms; more returns
+ * SR_ERR_TOO_LARGE and launches nothing.  The call allocates nothing and frees nothing.  The first call on a device
+ * looks up the array's device address (cudaGetSymbolAddress, with that device current) and sets the kernel's
+ * shared-memory limit; make that first call before any stream capture begins.  The array is shared by all calls on a
+ * device and keeps the previous call's contents; every block clears its part before use, so back-to-back calls on one
+ * stream are fine, but two calls that can overlap on the GPU (different streams or host threads) race on it and give
+ * wrong sums.  With 32 blocks instead of two per multiprocessor it is slower than sr_selection_gram on large inputs.
+ * A convenience of this library; the paper has no counterpart.
+ */
+int sr_selection_gram_static(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                             const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const sr_dims* d,
+                             uint32_t flags, void* stream);
 
 typedef struct sr_search_opts {
     double alpha;        /* fraction of the atoms to keep in the end, in (0, 1]                                   */

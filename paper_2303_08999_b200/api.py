@@ -17,11 +17,12 @@ LIB_PATH = os.path.join(_HERE, "libsr.so")
 
 SR_F32, SR_F16 = 0, 1
 SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16 = 1, 2, 4, 8, 16
-SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT = range(7)
+SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT, SR_ERR_TOO_LARGE = range(8)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
            "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival",
-           "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes")
+           "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes",
+           "sr_selection_gram_static")
 
 
 class sr_dims(ctypes.Structure):
@@ -68,6 +69,7 @@ def load_library() -> ctypes.CDLL:
         lib.sr_selection_gram_scratch_bytes.argtypes = [dp]
         lib.sr_selection_gram_scratch_bytes.restype = sz
         lib.sr_selection_gram.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, dp, u32, vp, sz, vp]
+        lib.sr_selection_gram_static.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, dp, u32, vp]
         lib.sr_selection_search_scratch_bytes.argtypes = [ctypes.c_int32]
         lib.sr_selection_search_scratch_bytes.restype = sz
         lib.sr_selection_search.argtypes = [vp, vp, vp, f64, ctypes.c_int32, ctypes.POINTER(sr_search_opts), vp, vp, vp, vp, vp, vp, sz, vp]

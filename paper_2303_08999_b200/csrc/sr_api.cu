@@ -237,6 +237,25 @@ int sr_selection_gram(const float* lr, const void* coef, int coef_dtype, const f
                                  nslots, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
 }
 
+int sr_selection_gram_static(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                             const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const sr_dims* d,
+                             uint32_t flags, void* stream)
+{
+    if (!lr || !coef || !dict || !target || !G || !b || !hh || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (d->D > selection_gram_static_max_atoms()) return SR_ERR_TOO_LARGE;       // beyond the built-in scratch
+    if (d->c > 16) return SR_ERR_UNSUPPORTED;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)SR_UPSAMPLE_BILINEAR) return SR_ERR_UNSUPPORTED;
+    if (samples && nsamples < 1) return SR_ERR_SHAPE;
+    if (!aligned(lr, 4) || !aligned(dict, 4) || !aligned(target, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4) ||
+        !aligned(G, 8) || !aligned(b, 8) || !aligned(hh, 8) || (samples && !aligned(samples, 8)))
+        return SR_ERR_ALIGN;
+    const Problem pb = make_problem(d, d->D, flags);
+    return launch_selection_gram_static(lr, coef, coef_dtype, dict, target, samples, nsamples, G, b, hh, pb,
+                                        (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
 size_t sr_selection_search_scratch_bytes(int32_t D) { return (D < 1 || D > 128) ? 0 : selection_search_scratch_bytes(D); }
 
 int sr_selection_search(const double* G, const double* b, const double* hh, double nrows, int32_t D,
@@ -267,6 +286,7 @@ const char* sr_status_string(int status)
     case SR_ERR_ALIGN: return "a pointer is misaligned";
     case SR_ERR_CUDA: return "a CUDA call or kernel launch failed";
     case SR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case SR_ERR_TOO_LARGE: return "the problem is larger than the library's built-in scratch memory";
     default: return "unknown status";
     }
 }

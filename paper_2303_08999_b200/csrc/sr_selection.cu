@@ -502,6 +502,48 @@ cudaError_t launch_selection_gram(const float* lr, const void* coef, int coef_dt
     return cudaGetLastError();
 }
 
+// ---- the Gram kernel without caller scratch --------------------------------------------------------------------------
+//
+// Some users of this library may not allocate device memory at the point where they want the Gram statistics: a
+// video pipeline that sizes all of its buffers once at start-up and runs under a fixed memory budget afterwards, a
+// plug-in inside a host application that owns the allocator, a service whose steady state must not call cudaMalloc
+// because that call synchronises the whole device and can fail long after start-up. For them the per-CTA fp64 slots of
+// selection_gram_kernel live in the array below instead of in memory the caller passes: kStaticGramSlots slots for at
+// most kStaticGramMaxD atoms, 32 x (80 x 80 + 80 + 8) doubles = 1 660 928 bytes that every device which loads the
+// library holds until the process exits. The array is shared by all calls and keeps what the last call left in it:
+// every CTA clears its own slot before it adds to it, and two calls whose kernels could run at the same time (two
+// streams, two host threads) must not both use this entry point, or they would sum into each other's slots.
+constexpr int kStaticGramSlots = 32;
+constexpr int kStaticGramMaxD = 80;
+static __device__ __align__(256) double g_gram_static_slots[kStaticGramSlots * (kStaticGramMaxD * kStaticGramMaxD + kStaticGramMaxD + 8)];
+
+int selection_gram_static_max_atoms() { return kStaticGramMaxD; }
+
+// Device address of the array above on the current device. In host code the array's name only stands for the symbol;
+// the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device while that device is current.
+static double* static_gram_slots()
+{
+    static double* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        double* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_gram_static_slots) != cudaSuccess) return nullptr;
+        cache[dev] = ptr;
+    }
+    return cache[dev];
+}
+
+cudaError_t launch_selection_gram_static(const float* lr, const void* coef, int coef_dtype, const float* dict, const float* target,
+                                         const int64_t* samples, int64_t nsamples, double* G, double* b, double* hh, const Problem& pb,
+                                         cudaStream_t st)
+{
+    if (pb.D > kStaticGramMaxD) return cudaErrorInvalidValue;
+    double* slots = static_gram_slots();
+    if (!slots) return cudaErrorUnknown;
+    return launch_selection_gram(lr, coef, coef_dtype, dict, target, samples, nsamples, G, b, hh, pb, slots, kStaticGramSlots, st);
+}
+
 size_t selection_search_scratch_bytes(int L) { return (size_t)L * L * sizeof(double); }
 
 cudaError_t launch_selection_search(const double* G, const double* b, const double* hh, double nrows, int L, const sr_search_opts& o,

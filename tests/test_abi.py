@@ -32,8 +32,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    seen = {sr.status_string(i) for i in range(7)}
-    assert len(seen) == 7 and sr.status_string(0) == "ok" and sr.status_string(99) == "unknown status"
+    seen = {sr.status_string(i) for i in range(8)}
+    assert len(seen) == 8 and sr.status_string(0) == "ok" and sr.status_string(99) == "unknown status"
 
 
 def _dims(**kw):
