@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the dictionary-regression hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg0|cfg1|cfg2|cfg3|cfg4]
 
 One step = one pass of the whole hot path over one frame batch of the workload (default: the
 1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. six library
@@ -20,6 +20,14 @@ slowest path); then the timed region, exactly K steps with events only around th
 (an event record costs about 3 us of stream time; the roofline kernel's duration comes from these).
 
 `--impl reference` times the CPU oracle (test infrastructure, fp64, as it stands) on the same workload.
+
+Workloads: cfg1 (the default; cfg2 is the same frame) prints the one JSON line of the benchmark contract. cfg0 (fp32
+coefficients, 128 x 128 output) and cfg3 (batch of four 4K frames) print one line of the same form. cfg4 is the shape
+sweep (LR 360 x 640, scale in {2,3,4}, D in {16,32,72,128}, k in {3,5,7}, s in {4,8,16}): one line per point and s, each
+with the per-path times and roofline fractions, the clocks seen during its timed region and the oracle timed on a
+small sample (`--points r3_D72_k5` restricts the sweep). Every path's roofline is the slowest of its bytes at the
+measured HBM bandwidth, its selection-network operations at the measured integer max/min rate and its multiply-adds
+at the measured fp32 rate (both rates are measured at start-up by the library's probe kernels).
 """
 from __future__ import annotations
 
@@ -84,35 +92,65 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
-# DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's
-# kernel on the default workload; figures and commands are in profiles/. None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.2, "select": 161.7, "compact": 25.7, "fused": 154.3, "global": 17.0}
+# DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's kernel on the
+# 1080p x4 frame (cfg1 / cfg2 only; figures and commands are in profiles/). None = not captured. The global-subset
+# figure is below its algorithmic bytes because the output frame (24.9 MB) is still in the 126 MB L2 when the kernel ends.
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.2, "select": 161.7, "compact": 25.7, "fused": 154.3, "global": 17.1}
 
 
-# Half-rate ALU-pipe lane operations per HR pixel of the two selection kernels (sorting-network max/min plus the
-# logic and address operations that share their pipe, counted from the networks in csrc/sr_select.cu and the select
-# role of csrc/sr_umma_impl.inc) and the B200 rate of that
-# pipe: 148 SMs x 64 lanes/clk x 1.965 GHz. The fused kernel works on packed binary16 pairs (two pixels per lane
-# operation): 315 max/min + 36 logic + 40 address operations per pixel, below its HBM time, so it is HBM-bound.
-ALU_OPS_PER_PIXEL = {"select": 630.0, "fused": 391.0}
-ALU_PEAK_GOPS = 148 * 64 * 1.965
+def selection_network_ops_per_pixel(path: str, D: int, s: int):
+    """Integer / packed max-min lane operations per HR pixel of the selection networks (csrc/sr_select.cu and the select
+    role of csrc/sr_umma_impl.inc): per group of eight planes a 19-exchange sort and a merge into the running list
+    (8 max + a 12-exchange bitonic merge for a list of 8; 8 max + 32 exchanges for a list of 16). The stand-alone kernel
+    works on 32-bit keys, one pixel per lane operation; the fused kernel on packed binary16 pairs, two pixels per lane
+    operation, plus 36 magnitude / logic and 40 address operations per 72 planes. These are the networks' own
+    operations: building the keys and the tails add about 45 % on the same pipe in the stand-alone kernel (ncu: ALU
+    pipe 84 % busy at 0.57 of this bound), instructions that are overhead to remove, not part of the bound."""
+    if s > 16 or path not in ("select", "fused"):
+        return 0.0
+    if path == "select":
+        # list of 4, 8 or 16 keys; groups of as many planes: sort (5 / 19 / 70 exchanges) + S max + merge (4 / 12 / 32 exchanges)
+        S, per_group = (4, 22.0) if s <= 4 else ((8, 70.0) if s <= 8 else (16, 220.0))
+        return per_group * ((D + S - 1) // S)
+    # fused: groups of eight planes against a list of 8 (s <= 8) or 16, two pixels per lane operation
+    per_group = 70.0 if s <= 8 else 110.0
+    return (per_group / 2 + 8.4) * ((D + 7) // 8)
 
 
-def path_roofline(wl, path: str, ms: float, hbm_peak: float, peak_kind: str, traffic_bytes_per_pixel):
-    """Roofline entry of one path: the slower of its bytes at HBM bandwidth and its selection ops at the ALU rate."""
+def fma_macs_per_pixel(wl, path: str):
+    """fp32 multiply-adds per HR pixel of the paths that run (or, by the survey's rule, are bounded) on the FMA pipe:
+    the small subset and compact forms (s k^2 + c k^2: assemble the filter from s atoms, then filter), and every
+    regression with fp32 coefficients (general kernel: D k^2 + c k^2)."""
+    kk = wl.k * wl.k
+    if wl.coef_dtype == "f32" and path in ("dense", "fused", "compact", "global"):
+        atoms = wl.D if path == "dense" else wl.s
+        return float(atoms * kk + wl.c * kk)
+    if path in ("compact", "global") and wl.s <= 8:
+        return float(wl.s * kk + wl.c * kk)
+    return 0.0
+
+
+def path_roofline(wl, path: str, ms: float, peaks: dict, traffic_bytes_per_pixel):
+    """Roofline entry of one path: the slowest of its bytes at HBM bandwidth, its selection operations at the integer
+    max/min rate and its multiply-adds at the fp32 rate; `frac` = that time / the measured time."""
     by = algorithmic_bytes_per_pixel(wl, path) * wl.npix
-    t_hbm = by / (hbm_peak * 1e9)
-    ops = ALU_OPS_PER_PIXEL.get(path, 0.0) * wl.npix if (wl.D == 72 and wl.s == 8) else 0.0
-    t_alu = ops / (ALU_PEAK_GOPS * 1e9)
+    ops = selection_network_ops_per_pixel(path, wl.D, wl.s) * wl.npix
+    macs = fma_macs_per_pixel(wl, path) * wl.npix
+    t = {"hbm": by / (peaks["hbm_gbs"] * 1e9), "alu": ops / peaks["alu_ops"], "fma": macs / peaks["fma_ops"]}
+    bound = max(t, key=lambda k: t[k])
     traffic = None if traffic_bytes_per_pixel is None else traffic_bytes_per_pixel * wl.npix
-    if t_alu > t_hbm:
-        ach = ops / (ms * 1e-3) / 1e9
-        return {"kernel": path, "bound": "alu", "achieved": ach, "peak": ALU_PEAK_GOPS, "unit": "Gop/s (max/min lanes)",
-                "frac": ach / ALU_PEAK_GOPS, "peak_kind": "derived: 148 SMs x 64 lanes/clk x 1.965 GHz", "traffic": traffic,
-                "hbm_frac": by / (ms * 1e-3) / 1e9 / hbm_peak}
-    ach = by / (ms * 1e-3) / 1e9
-    return {"kernel": path, "bound": "hbm", "achieved": ach, "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
-            "peak_kind": f"of {peak_kind}", "traffic": traffic}
+    sec = ms * 1e-3
+    if bound == "hbm":
+        out = {"bound": "hbm", "achieved": by / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"of {peaks['hbm_kind']}"}
+    elif bound == "alu":
+        out = {"bound": "alu", "achieved": ops / sec / 1e9, "peak": peaks["alu_ops"] / 1e9, "unit": "Gop/s (max/min lanes)",
+               "peak_kind": "measured at start-up by sr_probe_rate(0)"}
+    else:
+        out = {"bound": "fma", "achieved": macs / sec / 1e9, "peak": peaks["fma_ops"] / 1e9, "unit": "GMAC/s (fp32)",
+               "peak_kind": "measured at start-up by sr_probe_rate(1)"}
+    out.update({"kernel": path, "frac": out["achieved"] / out["peak"], "traffic": traffic, "roofline_us": t[bound] * 1e6,
+                "hbm_frac": by / sec / 1e9 / peaks["hbm_gbs"]})
+    return out
 
 
 class ClockSampler:
@@ -248,66 +286,46 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "MP/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(wl),
+        "config": workload_config(wl, 1),
         "cpu_baseline": {"value": value, "unit": "MP/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "MP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
 
 
-def workload_config(wl):
+def workload_config(wl, nsets: int):
     return {"workload": f"{wl.name}: LR {wl.n}x{wl.c}x{wl.h}x{wl.w} fp32, x{wl.scale} -> {wl.H}x{wl.W}, D={wl.D} atoms "
                         f"of {wl.k}x{wl.k}, coefficients {wl.coef_dtype} [n][D][H][W], top-s s={wl.s}",
             "paths_per_step": list(PATHS),
-            "l2": "coefficient tensor per frame is larger than the 126 MB L2 and three buffer sets rotate between steps"}
+            "l2": f"{nsets} coefficient buffer sets rotate between steps; together they are larger than twice the 126 MB L2"}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--workload", default="cfg1")
-    ap.add_argument("--paths", default=",".join(PATHS), help="comma-separated subset of the step's paths (profiling)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    active = tuple(p for p in PATHS if p in args.paths.split(","))
-    if "compact" in active and "select" not in active:
-        active = tuple(p for p in PATHS if p in active or p == "select")   # compact consumes select's outputs
+def rotating_sets(coef_bytes: int) -> int:
+    """Buffer sets to rotate through so that no coefficient read is served by the L2 (126 MB) of an earlier step."""
+    need = 2 * 126 * 1024 * 1024
+    return int(max(3, min(96, -(-need // max(1, coef_bytes)))))
 
-    import sr_inputs
-    wl = sr_inputs.CONFIGS[args.workload]
-    if args.impl == "reference":
-        run_reference(args, wl)
-        return
 
+def measure_peaks(sr):
+    hbm, kind = load_peaks()
+    return {"hbm_gbs": hbm, "hbm_kind": kind, "alu_ops": sr.sr_probe_rate(0), "fma_ops": sr.sr_probe_rate(1)}
+
+
+def run_workload(wl, args, active, peaks, dist, rank, world, local_rank, steps: int, warmup: int, with_e2e: bool, cpu_budget_s: float):
+    """Runs one workload on this rank and returns rank 0's JSON line (None on the other ranks)."""
     import numpy as np
     import torch
     import paper_2303_08999_b200 as sr
+    import sr_inputs
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    sr.load_library()
-
-    # ---- inputs: every rank owns its own frames (seed offset by rank); three rotating buffer sets
+    # ---- inputs: every rank owns its own frames (seed offset by rank); rotating buffer sets
     seed = rank_seed(sr_inputs.BASE_SEED, rank)
     lr, dict_, coef = sr_inputs.make_inputs(wl, seed)
     S = np.arange(0, wl.D, max(1, wl.D // wl.s), dtype=np.uint8)[: wl.s]
     gamma = np.linspace(0.75, 1.25, wl.s).astype(np.float32)
-    nsets = 3
-    h_lr = torch.from_numpy(lr).pin_memory()
-    h_coef = torch.from_numpy(coef).pin_memory()
+    nsets = rotating_sets(coef.nbytes)
+    h_lr = torch.from_numpy(lr).pin_memory() if with_e2e else torch.from_numpy(lr)
+    h_coef = torch.from_numpy(coef).pin_memory() if with_e2e else torch.from_numpy(coef)
     d_dict, d_S, d_gamma = (torch.from_numpy(a).cuda() for a in (dict_, S, gamma))
     sets = []
     for _ in range(nsets):
@@ -361,20 +379,20 @@ def main():
     sampler = ClockSampler(uuid) if rank == 0 else None
     if sampler:
         sampler.wait_first_sample()
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(sets[i % nsets])
     barrier()
 
     # ---- per-path pass (not the headline): the same K steps with an event between every call. It gives every path's
     # time and names the slowest one, whose kernel the roofline object describes.
     pass_events = []
-    for i in range(args.steps):
+    for i in range(steps):
         step(sets[i % nsets], pass_events)
     barrier()
     per_path_ms = {}
     per = len(PATHS) + 1
     for j, p in enumerate(PATHS):
-        ts = [pass_events[i * per + j].elapsed_time(pass_events[i * per + j + 1]) for i in range(args.steps)]
+        ts = [pass_events[i * per + j].elapsed_time(pass_events[i * per + j + 1]) for i in range(steps)]
         per_path_ms[p] = sum(ts) / len(ts)
     dominant_now = max(active, key=lambda p: per_path_ms[p])
 
@@ -385,7 +403,7 @@ def main():
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
     t_start.record()
-    for i in range(args.steps):
+    for i in range(steps):
         step(sets[i % nsets], events, only=dominant_now)
     t_end.record()
     barrier()
@@ -396,19 +414,19 @@ def main():
     if sr.sr_device_status() != 0:
         raise SystemExit("device status word reports an expired wait")
     elapsed_ms = max_over_ranks(elapsed_ms, dist, "cuda")
-    assert len(events) == 2 * args.steps
-    ts = [events[2 * i].elapsed_time(events[2 * i + 1]) for i in range(args.steps)]
+    assert len(events) == 2 * steps
+    ts = [events[2 * i].elapsed_time(events[2 * i + 1]) for i in range(steps)]
     per_path_ms[dominant_now] = sum(ts) / len(ts)               # the roofline kernel's time comes from the timed region
 
     # ---- end to end through the public API with host buffers: pinned H2D of the step's inputs, D2H of its results
     e2e = None
-    if not args.no_e2e:
+    if with_e2e:
         # Two figures.  `value`: a stream of frames through HostPipeline (step i+1's inputs travel while step i's
         # results do; every step still copies all its inputs in and all its results out inside the timed region).
         # `serial_value`: one step at a time on one stream, copy in -> kernels -> copy out.
         from paper_2303_08999_b200.hostpipe import HostPipeline
         h_out = {p: torch.empty(shape_out, dtype=torch.float32).pin_memory() for p in outs}
-        e2e_steps = max(3, min(args.steps, 10))
+        e2e_steps = max(3, min(steps, 10))
         host_in = {"lr": h_lr, "coef": h_coef}
         pipe = HostPipeline({"lr": (tuple(h_lr.shape), h_lr.dtype), "coef": (tuple(h_coef.shape), h_coef.dtype)},
                             {p: (shape_out, torch.float32) for p in outs}, depth=2)
@@ -444,39 +462,96 @@ def main():
                "how": "HostPipeline, depth 2: copy-in, kernels and copy-out on three streams",
                "serial_value": whole_job_value(world, wl.npix, e2e_steps, ms_serial)}
 
+    del sets, outs, idx, sel
+    torch.cuda.empty_cache()
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
 
-    peak, peak_kind = load_peaks()
+    traffic = NCU_TRAFFIC_BYTES_PER_PIXEL if wl.name in ("cfg1", "cfg2") else {}
     paths = {}
     for p in active:
         by = algorithmic_bytes_per_pixel(wl, p) * wl.npix
         gbs = by / (per_path_ms[p] * 1e-3) / 1e9
         paths[p] = {"ms": per_path_ms[p], "mp_per_s": wl.npix / (per_path_ms[p] * 1e-3) / 1e6,
                     "frames_per_s": wl.n / (per_path_ms[p] * 1e-3), "algorithmic_bytes": by, "achieved_gbs": gbs,
-                    "frac_of_hbm": gbs / peak}
-    dominant = dominant_now
-    roofline = path_roofline(wl, dominant, per_path_ms[dominant], peak, peak_kind, NCU_TRAFFIC_BYTES_PER_PIXEL.get(dominant))
-    for p in active:
-        paths[p]["roofline"] = path_roofline(wl, p, per_path_ms[p], peak, peak_kind, NCU_TRAFFIC_BYTES_PER_PIXEL.get(p))
+                    "frac_of_hbm": gbs / peaks["hbm_gbs"],
+                    "roofline": path_roofline(wl, p, per_path_ms[p], peaks, traffic.get(p))}
+    roofline = path_roofline(wl, dominant_now, per_path_ms[dominant_now], peaks, traffic.get(dominant_now))
 
     cpu = None
-    if not args.no_cpu_baseline:
-        cpu = time_oracle(wl, lr, dict_, coef, S, gamma)
+    if cpu_budget_s > 0:
+        cpu = time_oracle(wl, lr, dict_, coef, S, gamma, budget_s=cpu_budget_s)
 
-    line = {
-        "metric": METRIC, "value": whole_job_value(world, wl.npix, args.steps, elapsed_ms), "unit": "MP/s",
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
+    return {
+        "metric": METRIC, "value": whole_job_value(world, wl.npix, steps, elapsed_ms), "unit": "MP/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": elapsed_ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate, f16 coefficients"
-        if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": dict(workload_config(wl), paths_per_step=list(active)),
+        if wl.coef_dtype == "f16" else "f32", "data": "synthetic", "config": dict(workload_config(wl, nsets), paths_per_step=list(active)),
         "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
         "paths": paths,
+        "peaks": {"hbm_gbs": peaks["hbm_gbs"], "hbm": f"of {peaks['hbm_kind']}", "int_maxmin_gops": peaks["alu_ops"] / 1e9,
+                  "fp32_fma_gmacs": peaks["fma_ops"] / 1e9, "how": "HBM: MEASURED_PEAKS.json; pipes: sr_probe_rate at start-up"},
         "paths_timing": "pass of K steps with an event between every call, before the timed region; the roofline "
                         "kernel's time is from the events inside the timed region",
     }
-    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--points", default="", help="cfg4 only: comma-separated substrings of point names, e.g. r3_D72_k5")
+    ap.add_argument("--paths", default=",".join(PATHS), help="comma-separated subset of the step's paths (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    sweep = args.workload == "cfg4"
+    steps = args.steps if args.steps is not None else (20 if sweep else (30 if args.workload == "cfg3" else 300))
+    warmup = args.warmup if args.warmup is not None else (3 if sweep or args.workload == "cfg3" else 10)
+    if args.impl == "ours":
+        warmup = max(warmup, 3)
+    args.steps, args.warmup = steps, warmup
+    active = tuple(p for p in PATHS if p in args.paths.split(","))
+    if "compact" in active and "select" not in active:
+        active = tuple(p for p in PATHS if p in active or p == "select")   # compact consumes select's outputs
+
+    import sr_inputs
+    from dataclasses import replace
+    if sweep:
+        want = [w for w in args.points.split(",") if w]
+        wls = [replace(p, s=s) for p in sr_inputs.cfg4_points() for s in (4, 8, 16)
+               if s <= p.D and (not want or any(w in p.name for w in want))]
+    else:
+        wls = [sr_inputs.CONFIGS[args.workload]]
+    if args.impl == "reference":
+        run_reference(args, sr_inputs.CONFIGS[args.workload])    # the sweep's reference arm times its anchor point
+        return
+
+    import torch
+    import paper_2303_08999_b200 as sr
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    sr.load_library()
+    peaks = measure_peaks(sr)
+    default_line = args.workload in ("cfg1", "cfg2")
+    for wl in wls:
+        line = run_workload(wl, args, active, peaks, dist, rank, world, local_rank, steps, warmup,
+                            with_e2e=default_line and not args.no_e2e,
+                            cpu_budget_s=0.0 if args.no_cpu_baseline else (1.0 if sweep else 20.0))
+        if line is not None:
+            print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 

@@ -225,6 +225,45 @@ const char* sr_status_string(int status);
 int sr_device_status(void* stream, int* out_status);
 
 /*
+ * Tile-shape search (Section III-B, restated for this library).  The paper prunes the space of thread-block shapes
+ * of its filtering kernel with resource constraints (Eq. 11-12) and searches the rest by measured latency.  Here the
+ * tunable shape of a regression launch is: which kernel takes it (first or second tensor-core layout, the FMA-pipe
+ * subset kernel), the tile height, and the rows per pipeline step; the legal set follows from the shared memory per
+ * thread block, the tensor-memory columns and the stage count, and is small enough to time exhaustively.
+ * sr_tune_dense / sr_tune_selected take the arguments of the call they tune plus `reps`, run every legal shape
+ * (one warm-up launch, then `reps` timed launches between two CUDA events) on the caller's own buffers, and record the
+ * fastest for this problem shape (n, c, h, w, scale, k, D, s, flags, coefficient type); later calls of
+ * sr_dict_regress_dense / sr_dict_regress_selected with the same shape use it.  They synchronise `stream`, overwrite
+ * `out`, and are meant to be called once per shape at start-up; inputs that are not larger than the L2 cache are timed
+ * warm.  The per-pixel arithmetic does not depend on the tile shape, so results for one kernel are the same bits for
+ * every shape.  *result (may be NULL) receives the choice.  sr_tune_reset forgets every recorded shape.
+ */
+typedef struct sr_tune_result {
+    int32_t kernel;        /* 0 general FMA kernel, 1 first tensor-core layout, 2 second tensor-core layout, 3 subset kernel */
+    int32_t tile_rows;     /* tile height (kernels 2 and 3; 0 otherwise)                                               */
+    int32_t rows_per_step; /* tile rows per pipeline step (kernel 2; 0 otherwise)                                      */
+    int32_t candidates;    /* launch shapes that were legal and timed                                                   */
+    float best_us;         /* time per launch of the recorded shape                                                     */
+    float default_us;      /* time per launch of the shape the host rules pick without tuning                           */
+} sr_tune_result;
+int sr_tune_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out, const sr_dims* d,
+                  uint32_t flags, int reps, void* stream, sr_tune_result* result);
+int sr_tune_selected(const float* lr, const void* coef_or_sel, int coef_dtype, const uint8_t* idx, const float* gamma,
+                     const float* dict, float* out, const sr_dims* d, int s, uint32_t flags, int reps, void* stream,
+                     sr_tune_result* result);
+void sr_tune_reset(void);
+
+/*
+ * Sustained issue rate of an arithmetic pipe of the current device, for the roofline of the kernels that are bound by
+ * one (the selection networks by integer max/min, the general and subset regressions by fp32 multiply-add):
+ * kind 0 = integer max/min, kind 1 = fp32 multiply-add.  Runs a register-only kernel a few times on `stream`,
+ * synchronises it, and writes lane operations per second to *lane_ops_per_s (HOST pointer).  `scratch8` is 8 bytes of
+ * device memory whose first int is read (any value) and which is otherwise left alone.  Introspection for benchmarks;
+ * the paper has no counterpart.
+ */
+int sr_probe_rate(int kind, void* scratch8, double* lane_ops_per_s, void* stream);
+
+/*
  * Cycle budget of every device-side wait (mbarrier waits for copies, tensor-core results and tile hand-overs) in
  * the launches that follow, process-wide; the default is 2^31 SM cycles, about a second.  A wait that runs out
  * makes its thread block stop, wait briefly for its copies and tensor-core operations in flight, free its tensor

@@ -22,7 +22,7 @@ SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA,
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
            "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival",
            "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes",
-           "sr_selection_gram_static")
+           "sr_selection_gram_static", "sr_probe_rate", "sr_tune_dense", "sr_tune_selected", "sr_tune_reset")
 
 
 class sr_dims(ctypes.Structure):
@@ -32,6 +32,11 @@ class sr_dims(ctypes.Structure):
 class sr_search_opts(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_double), ("delta_alpha", ctypes.c_double), ("eps", ctypes.c_double), ("lambda0", ctypes.c_double),
                 ("tol", ctypes.c_double), ("max_sweeps", ctypes.c_int32), ("max_bisect", ctypes.c_int32), ("max_steps", ctypes.c_int32)]
+
+
+class sr_tune_result(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_int32), ("tile_rows", ctypes.c_int32), ("rows_per_step", ctypes.c_int32),
+                ("candidates", ctypes.c_int32), ("best_us", ctypes.c_float), ("default_us", ctypes.c_float)]
 
 
 class SrError(RuntimeError):
@@ -60,6 +65,7 @@ def load_library() -> ctypes.CDLL:
         lib.sr_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
         for name in EXPORTS:
             getattr(lib, name).restype = i32
+        lib.sr_tune_reset.restype = None
         lib.sr_launch_count.argtypes = []
         lib.sr_launch_count.restype = ctypes.c_int64
         lib.sr_set_wait_limit.argtypes = [ctypes.c_int64]
@@ -69,6 +75,11 @@ def load_library() -> ctypes.CDLL:
         lib.sr_selection_gram_scratch_bytes.argtypes = [dp]
         lib.sr_selection_gram_scratch_bytes.restype = sz
         lib.sr_selection_gram.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, dp, u32, vp, sz, vp]
+        tp = ctypes.POINTER(sr_tune_result)
+        lib.sr_tune_dense.argtypes = [vp, vp, i32, vp, vp, dp, u32, i32, vp, tp]
+        lib.sr_tune_selected.argtypes = [vp, vp, i32, vp, vp, vp, vp, dp, i32, u32, i32, vp, tp]
+        lib.sr_tune_reset.argtypes = []
+        lib.sr_probe_rate.argtypes = [i32, vp, ctypes.POINTER(ctypes.c_double), vp]
         lib.sr_selection_gram_static.argtypes = [vp, vp, i32, vp, vp, vp, i64, vp, vp, vp, dp, u32, vp]
         lib.sr_selection_search_scratch_bytes.argtypes = [ctypes.c_int32]
         lib.sr_selection_search_scratch_bytes.restype = sz
@@ -263,3 +274,49 @@ def sr_selection_search(G, b, hh, nrows: float, alpha: float, delta_alpha: float
     if n < 0:
         raise SrError(SR_ERR_UNSUPPORTED, "sr_selection_search: a re-fit met a singular matrix")
     return idx[:n], gamma[:n], trace[: int(steps.item())]
+
+
+def sr_probe_rate(kind: int) -> float:
+    """Sustained lane operations per second of integer max/min (kind 0) or fp32 multiply-add (kind 1) on the current device."""
+    scratch = torch.zeros(2, dtype=torch.int32, device="cuda")
+    v = ctypes.c_double(0.0)
+    _check(load_library().sr_probe_rate(kind, _ptr(scratch), ctypes.byref(v), _stream()), "sr_probe_rate")
+    return float(v.value)
+
+
+def _tune_dict(res: sr_tune_result) -> dict:
+    names = {0: "general", 1: "first tensor-core layout", 2: "second tensor-core layout", 3: "subset (FMA pipe)"}
+    return {"kernel": names.get(res.kernel, str(res.kernel)), "tile_rows": res.tile_rows, "rows_per_step": res.rows_per_step,
+            "candidates": res.candidates, "best_us": res.best_us, "default_us": res.default_us}
+
+
+def sr_tune_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, reps: int = 5) -> dict:
+    """Tile-shape search for sr_dict_regress_dense on these buffers; later calls with the same shape use the result."""
+    lr, dict_ = _dev(lr, torch.float32, "lr"), _dev(dict_, torch.float32, "dict")
+    code = _coef_code(coef)
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float16 if (flags & SR_OUT_F16) else torch.float32, device=lr.device)
+    d = sr_dims(n, c, h, w, scale, k, D)
+    res = sr_tune_result()
+    _check(load_library().sr_tune_dense(_ptr(lr), _ptr(coef), code, _ptr(dict_), _ptr(out), ctypes.byref(d), flags, reps, _stream(),
+                                        ctypes.byref(res)), "sr_tune_dense")
+    return _tune_dict(res)
+
+
+def sr_tune_selected(lr, coef_or_sel, idx, gamma, dict_, scale: int, k: int, s: int, flags: int = 0, reps: int = 5) -> dict:
+    """Tile-shape search for sr_dict_regress_selected on these buffers."""
+    lr, dict_ = _dev(lr, torch.float32, "lr"), _dev(dict_, torch.float32, "dict")
+    code = _coef_code(coef_or_sel)
+    n, c, h, w = lr.shape
+    D = dict_.shape[0]
+    out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float16 if (flags & SR_OUT_F16) else torch.float32, device=lr.device)
+    d = sr_dims(n, c, h, w, scale, k, D)
+    res = sr_tune_result()
+    _check(load_library().sr_tune_selected(_ptr(lr), _ptr(coef_or_sel), code, _ptr(idx), _ptr(gamma), _ptr(dict_), _ptr(out),
+                                           ctypes.byref(d), s, flags, reps, _stream(), ctypes.byref(res)), "sr_tune_selected")
+    return _tune_dict(res)
+
+
+def sr_tune_reset() -> None:
+    load_library().sr_tune_reset()

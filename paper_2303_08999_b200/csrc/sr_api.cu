@@ -2,6 +2,10 @@
 #include <math.h>
 
 #include <atomic>
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <vector>
 
 #include "sr_common.cuh"
 #include "sr_regress_subset.cuh"
@@ -113,6 +117,162 @@ static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 // on the 1080p sweep points (dense, D = 16 / 32 / 72 / 128; k = 3 / 5 / 7).
 static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 || (pb.k == 7 && pb.D <= 32); }
 
+// ---- which kernel runs a regression, and in which launch shape ----------------------------------------------------------
+//
+// Every regression call goes through run_regress. Without an entry in the tuning table it takes the kernel and shape
+// the host rules pick; sr_tune_dense / sr_tune_selected time every legal alternative on the caller's buffers and record
+// the fastest for that problem shape (the block-shape search of Section III-B, restated for this library: the legal
+// set comes from shared-memory, tensor-memory and stage-count constraints instead of register-file and warp-scheduler
+// limits, and it is small enough to be timed exhaustively instead of by Bayesian optimisation).
+enum RegressKernel { kKernelGeneral = 0, kKernelFirstLayout = 1, kKernelSecondLayout = 2, kKernelSubset = 3 };
+
+struct TuneChoice {
+    int kernel = -1;      // -1: host rules
+    TcTuning tc;          // second layout: tile height and rows per pipeline step
+    int sub_th = 0;       // subset kernel: tile height
+};
+
+typedef std::tuple<int, int, int, int, int, int, int, int, int, uint32_t, int> TuneKey;
+
+static TuneKey tune_key(int mode, int coef_dtype, const Problem& pb)
+{
+    return TuneKey(mode, pb.n, pb.c, pb.h, pb.w, pb.r, pb.k, pb.D, pb.s, pb.flags, coef_dtype);
+}
+
+static std::mutex g_tune_mu;
+static std::map<TuneKey, TuneChoice> g_tune_table;
+
+static bool tune_lookup(const TuneKey& key, TuneChoice& out)
+{
+    std::lock_guard<std::mutex> lock(g_tune_mu);
+    auto it = g_tune_table.find(key);
+    if (it == g_tune_table.end()) return false;
+    out = it->second;
+    return true;
+}
+
+static int selected_mode(const uint8_t* idx, uint32_t flags)
+{
+    if (flags & SR_IDX_GLOBAL) return kModeGlobal;
+    if (flags & SR_COEF_COMPACT) return kModeCompact;
+    return idx ? kModeIdx : kModeFusedSelect;
+}
+
+struct RegressArgs {
+    int mode;
+    const float* lr;
+    const void* coef;
+    int coef_dtype;
+    const uint8_t* idx;
+    const float* gamma;
+    const float* dict;
+    float* out;
+    Problem pb;
+    cudaStream_t st;
+};
+
+static bool kernel_supported(int kernel, const RegressArgs& a)
+{
+    const bool idx_vec_ok = !a.idx || a.mode == kModeGlobal || ((reinterpret_cast<uintptr_t>(a.idx) & 15) == 0);   // 16-byte reads
+    switch (kernel) {
+    case kKernelSubset: return regress_subset_supported(a.mode, a.coef, a.coef_dtype, a.out, a.pb);
+    case kKernelSecondLayout: return regress_tc_supported(a.mode, a.coef, a.coef_dtype, a.pb);
+    case kKernelFirstLayout: return idx_vec_ok && umma_supported(a.mode, a.coef, a.coef_dtype, a.pb);
+    default: return true;
+    }
+}
+
+// The host rules: small global subsets on the FMA-pipe subset kernel; the second tensor-core layout for the other
+// global subsets and for dense launches with few atoms; the first layout for the rest it supports; else the general kernel.
+static int default_kernel(const RegressArgs& a)
+{
+    if (kernel_supported(kKernelSubset, a)) return kKernelSubset;
+    const bool first = kernel_supported(kKernelFirstLayout, a), second = kernel_supported(kKernelSecondLayout, a);
+    if (second && (a.mode == kModeGlobal || dense_prefers_second_layout(a.pb) || !first)) return kKernelSecondLayout;
+    if (first) return kKernelFirstLayout;
+    return kKernelGeneral;
+}
+
+static cudaError_t run_kernel(const TuneChoice& c, const RegressArgs& a)
+{
+    switch (c.kernel) {
+    case kKernelSubset: return launch_regress_subset(a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st, c.sub_th);
+    case kKernelSecondLayout: return launch_regress_tc(a.mode, a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st, c.tc);
+    case kKernelFirstLayout: return launch_regress_umma(a.mode, a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st);
+    default: return launch_regress_fma(a.mode, a.lr, a.coef, a.coef_dtype, a.idx, a.gamma, a.dict, a.out, a.pb, a.st);
+    }
+}
+
+static cudaError_t run_regress(const RegressArgs& a)
+{
+    TuneChoice c;
+    if (tune_lookup(tune_key(a.mode, a.coef_dtype, a.pb), c) && kernel_supported(c.kernel, a)) return run_kernel(c, a);
+    c = TuneChoice{};
+    c.kernel = default_kernel(a);
+    return run_kernel(c, a);
+}
+
+// Times `reps` launches of one candidate after one warm-up launch; microseconds per launch, negative on error.
+static float time_candidate(const TuneChoice& c, const RegressArgs& a, int reps, cudaEvent_t e0, cudaEvent_t e1)
+{
+    if (run_kernel(c, a) != cudaSuccess) return -1.f;
+    if (cudaEventRecord(e0, a.st) != cudaSuccess) return -1.f;
+    for (int i = 0; i < reps; ++i)
+        if (run_kernel(c, a) != cudaSuccess) return -1.f;
+    if (cudaEventRecord(e1, a.st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) return -1.f;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) return -1.f;
+    return ms * 1e3f / (float)reps;
+}
+
+static int tune_shape(const RegressArgs& a, int reps, sr_tune_result* res)
+{
+    if (reps < 1) reps = 1;
+    std::vector<TuneChoice> cands;
+    if (kernel_supported(kKernelFirstLayout, a)) { TuneChoice c; c.kernel = kKernelFirstLayout; cands.push_back(c); }
+    if (kernel_supported(kKernelSecondLayout, a)) {
+        TcTuning shapes[64];
+        const int n = regress_tc_candidates(a.mode, a.pb, shapes, 64);
+        for (int i = 0; i < n; ++i) { TuneChoice c; c.kernel = kKernelSecondLayout; c.tc = shapes[i]; cands.push_back(c); }
+    }
+    if (kernel_supported(kKernelSubset, a)) {
+        int ths[8];
+        const int n = regress_subset_candidates(a.pb, ths, 8);
+        for (int i = 0; i < n; ++i) { TuneChoice c; c.kernel = kKernelSubset; c.sub_th = ths[i]; cands.push_back(c); }
+    }
+    if (cands.empty()) { TuneChoice c; c.kernel = kKernelGeneral; cands.push_back(c); }
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess) return SR_ERR_CUDA;
+    if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return SR_ERR_CUDA; }
+    TuneChoice def;
+    def.kernel = default_kernel(a);
+    const float def_us = time_candidate(def, a, reps, e0, e1);
+    int best = -1;
+    float best_us = 0.f;
+    for (size_t i = 0; i < cands.size(); ++i) {
+        const float us = time_candidate(cands[i], a, reps, e0, e1);
+        if (us > 0.f && (best < 0 || us < best_us)) { best = (int)i; best_us = us; }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (best < 0 || def_us < 0.f) return SR_ERR_CUDA;
+    TuneChoice pick = cands[best];
+    if (def_us <= best_us) { pick = def; best_us = def_us; }        // the host rules' own choice stays unless something beat it
+    {
+        std::lock_guard<std::mutex> lock(g_tune_mu);
+        g_tune_table[tune_key(a.mode, a.coef_dtype, a.pb)] = pick;
+    }
+    if (res) {
+        res->kernel = pick.kernel;
+        res->tile_rows = pick.kernel == kKernelSecondLayout ? pick.tc.th : (pick.kernel == kKernelSubset ? pick.sub_th : 0);
+        res->rows_per_step = pick.kernel == kKernelSecondLayout ? pick.tc.group : 0;
+        res->candidates = (int32_t)cands.size();
+        res->best_us = best_us;
+        res->default_us = def_us;
+    }
+    return SR_OK;
+}
+
 } // namespace sr
 
 using namespace sr;
@@ -149,16 +309,21 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
     if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
     if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
-    const Problem pb = make_problem(d, d->D, flags);
-    cudaError_t err;
-    const bool first_ok = umma_supported(kModeDense, coef, coef_dtype, pb);
-    if (regress_tc_supported(kModeDense, coef, coef_dtype, pb) && (dense_prefers_second_layout(pb) || !first_ok))
-        err = launch_regress_tc(kModeDense, lr, coef, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
-    else if (first_ok)
-        err = launch_regress_umma(kModeDense, lr, coef, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
-    else
-        err = launch_regress_fma(kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, pb, (cudaStream_t)stream);
-    return err == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+    const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
+    return run_regress(a) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_tune_dense(const float* lr, const void* coef, int coef_dtype, const float* dict, float* out, const sr_dims* d,
+                  uint32_t flags, int reps, void* stream, sr_tune_result* result)
+{
+    if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
+        return SR_ERR_ALIGN;
+    const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
+    return tune_shape(a, reps, result);
 }
 
 int sr_dict_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, const sr_dims* d, int s, uint32_t flags,
@@ -191,22 +356,32 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
         !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
-    const Problem pb = make_problem(d, s, flags);
-    int mode;
-    if (flags & SR_IDX_GLOBAL) mode = kModeGlobal;
-    else if (flags & SR_COEF_COMPACT) mode = kModeCompact;
-    else mode = idx ? kModeIdx : kModeFusedSelect;
-    cudaError_t err;
-    const bool idx_vec_ok = !idx || (flags & SR_IDX_GLOBAL) || ((reinterpret_cast<uintptr_t>(idx) & 15) == 0);   // 16-byte reads
-    if (regress_subset_supported(mode, coef_or_sel, coef_dtype, out, pb))
-        err = launch_regress_subset(lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
-    else if (regress_tc_supported(mode, coef_or_sel, coef_dtype, pb))
-        err = launch_regress_tc(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
-    else if (idx_vec_ok && umma_supported(mode, coef_or_sel, coef_dtype, pb))
-        err = launch_regress_umma(mode, lr, coef_or_sel, idx, gamma, dict, out, pb, (cudaStream_t)stream);
-    else
-        err = launch_regress_fma(mode, lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, pb, (cudaStream_t)stream);
-    return err == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+    const RegressArgs a{selected_mode(idx, flags), lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, make_problem(d, s, flags), (cudaStream_t)stream};
+    return run_regress(a) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_tune_selected(const float* lr, const void* coef_or_sel, int coef_dtype, const uint8_t* idx, const float* gamma,
+                     const float* dict, float* out, const sr_dims* d, int s, uint32_t flags, int reps, void* stream,
+                     sr_tune_result* result)
+{
+    if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
+    if (s < 1 || s > d->D) return SR_ERR_SHAPE;
+    if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
+    if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
+        !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
+        return SR_ERR_ALIGN;
+    const RegressArgs a{selected_mode(idx, flags), lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, make_problem(d, s, flags), (cudaStream_t)stream};
+    return tune_shape(a, reps, result);
+}
+
+void sr_tune_reset(void)
+{
+    std::lock_guard<std::mutex> lock(g_tune_mu);
+    g_tune_table.clear();
 }
 
 size_t sr_selection_gram_scratch_bytes(const sr_dims* d)
@@ -292,6 +467,14 @@ const char* sr_status_string(int status)
 }
 
 int64_t sr_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+int sr_probe_rate(int kind, void* scratch8, double* lane_ops_per_s, void* stream)
+{
+    if (!scratch8 || !lane_ops_per_s) return SR_ERR_NULL;
+    if (kind != 0 && kind != 1) return SR_ERR_UNSUPPORTED;
+    if (!aligned(scratch8, 4)) return SR_ERR_ALIGN;
+    return probe_rate(kind, static_cast<int*>(scratch8), lane_ops_per_s, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
 
 int64_t sr_set_wait_limit(int64_t cycles)
 {

@@ -54,6 +54,9 @@ int sm_count();
 // Adds to the process-wide count of kernels launched (read back by sr_launch_count).
 void count_launches(int n);
 
+// Issue-rate probe (sr_probe.cu): kind 0 integer max/min, 1 fp32 multiply-add; lane operations per second.
+cudaError_t probe_rate(int kind, int* scratch2, double* lane_ops_per_s, cudaStream_t st);
+
 // Launchers. Each returns a cudaError_t from the launch.
 cudaError_t launch_bicubic(const float* lr, float* hr, const Problem& pb, cudaStream_t st);
 cudaError_t launch_regress_fma(int mode, const float* lr, const void* coef, int coef_dtype, const uint8_t* idx,

@@ -226,14 +226,13 @@ const DeviceInfo& device_info()
 
 constexpr int kStaticReserve = 2048;   // static shared memory + the per-CTA system reservation
 
-int g_forced_th = 0;
 
 // Tile height: the tiles are dealt round-robin to the resident CTAs, a warp takes every eighth row of a tile, so a
 // tile costs ceil(th / 8) row passes plus its up-sampled tile (th + k - 1 rows) and three CTA-wide barriers; the
 // launch takes as long as the CTA with the most tiles. Units: warp instructions. The per-tile term is set from
 // timings (1080p x4, s = 8: 59 / 58 / 51 us at th = 8 / 16 / 24): the tallest tile wins although it divides the
 // frame less evenly, because a tile's fixed work is about as long as sixteen rows of filtering.
-int choose_th(const Problem& pb, int nq, size_t& smem_bytes, int& ctas)
+int choose_th(const Problem& pb, int nq, size_t& smem_bytes, int& ctas, int g_forced_th = 0)
 {
     const DeviceInfo& di = device_info();
     const int per_cta = di.smem_sm / 2 - kStaticReserve;
@@ -299,7 +298,17 @@ cudaError_t launch_q(const SubParams& prm, int ctas, size_t smem, cudaStream_t s
 
 } // namespace
 
-void regress_subset_force_tile_height(int th) { g_forced_th = (th == 8 || th == 16 || th == 24) ? th : 0; }
+// Tile heights the problem admits (shared memory of two CTAs per SM); the tile-shape search times these.
+int regress_subset_candidates(const Problem& pb, int* ths, int max_out)
+{
+    int n = 0;
+    for (int th = 24; th >= 8; th -= 8) {
+        size_t smem;
+        int ctas;
+        if (choose_th(pb, pb.s <= 4 ? 4 : 8, smem, ctas, th) == th && n < max_out) ths[n++] = th;
+    }
+    return n;
+}
 
 bool regress_subset_supported(int mode, const void* coef, int coef_dtype, const void* out, const Problem& pb)
 {
@@ -315,12 +324,12 @@ bool regress_subset_supported(int mode, const void* coef, int coef_dtype, const 
 }
 
 cudaError_t launch_regress_subset(const float* lr, const void* coef, const uint8_t* idx, const float* gamma, const float* dict,
-                                  float* out, const Problem& pb, cudaStream_t st)
+                                  float* out, const Problem& pb, cudaStream_t st, int th_forced)
 {
     SubParams prm{};
     size_t smem = 0;
     int ctas = 0;
-    const int th = choose_th(pb, pb.s <= 4 ? 4 : 8, smem, ctas);
+    const int th = choose_th(pb, pb.s <= 4 ? 4 : 8, smem, ctas, th_forced);
     if (th == 0) return cudaErrorNotSupported;
     plan_geom(prm.g, pb, th, lr);
     prm.lr = lr; prm.dict = dict; prm.out = out; prm.idx = idx; prm.gamma = gamma;

@@ -9,9 +9,9 @@ namespace sr {
 bool regress_subset_supported(int mode, const void* coef, int coef_dtype, const void* out, const Problem& pb);
 
 cudaError_t launch_regress_subset(const float* lr, const void* coef, const uint8_t* idx, const float* gamma, const float* dict,
-                                  float* out, const Problem& pb, cudaStream_t st);
+                                  float* out, const Problem& pb, cudaStream_t st, int th_forced = 0);
 
-// Tile height of the launches that follow: 8, 16 or 24; 0 = the host's cost model (tile-shape search).
-void regress_subset_force_tile_height(int th);
+// Tile heights (8, 16, 24) the problem admits; returns how many were written.
+int regress_subset_candidates(const Problem& pb, int* ths, int max_out);
 
 } // namespace sr

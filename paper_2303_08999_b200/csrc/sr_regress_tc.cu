@@ -661,9 +661,7 @@ Plan make_plan_k(int mode, const Problem& pb, const TcTuning& tune)
 // hi and lo halves stacked along K while the atoms are few (the extra MMAs are cheap then); side by side along N otherwise
 bool use_hilo(int natoms) { return natoms > 32; }
 
-TcTuning g_tune;   // zeros: everything chosen by the cost model
-
-Plan make_plan(int mode, const Problem& pb)
+Plan make_plan(int mode, const Problem& pb, const TcTuning& g_tune)
 {
     int natoms, gather;
     contraction_shape(mode, pb, natoms, gather);
@@ -714,10 +712,21 @@ cudaError_t launch_k(const CUtensorMap& map_lead, const TcParams& prm, const Pla
 
 } // namespace
 
-void regress_tc_set_tuning(const TcTuning& t)
+// Every legal launch shape of this path for the problem: tile heights 4..16 x rows per pipeline step {1, 2, 4}, kept
+// when the shared memory of a CTA (stages, B operand, up-sampling buffers), its tensor-memory columns (two groups of
+// accumulators) and the stage count (>= 2) allow it. The tile-shape search times these.
+int regress_tc_candidates(int mode, const Problem& pb, TcTuning* out, int max_out)
 {
-    g_tune.th = (t.th >= 4 && t.th <= kMaxTH) ? t.th : 0;
-    g_tune.group = (t.group == 1 || t.group == 2 || t.group == 4) ? t.group : 0;
+    int n = 0;
+    for (int th = kMaxTH; th >= 4; --th)
+        for (int group = kMaxGroupRows; group >= 1; group >>= 1) {
+            TcTuning t;
+            t.th = th;
+            t.group = group;
+            const Plan pl = make_plan(mode, pb, t);
+            if (pl.ok && pl.th == th && pl.group == group && n < max_out) out[n++] = t;
+        }
+    return n;
 }
 
 bool regress_tc_supported(int mode, const void* coef, int coef_dtype, const Problem& pb)
@@ -729,13 +738,13 @@ bool regress_tc_supported(int mode, const void* coef, int coef_dtype, const Prob
     if (pb.n > 65535) return false;
     const DeviceInfo& di = device_info();
     if (!di.ok || di.cc_major != 10) return false;
-    return make_plan(mode, pb).ok;
+    return make_plan(mode, pb, TcTuning{}).ok;
 }
 
 cudaError_t launch_regress_tc(int mode, const float* lr, const void* coef, const uint8_t* idx, const float* gamma,
-                              const float* dict, float* out, const Problem& pb, cudaStream_t st)
+                              const float* dict, float* out, const Problem& pb, cudaStream_t st, const TcTuning& tune)
 {
-    const Plan pl = make_plan(mode, pb);
+    const Plan pl = make_plan(mode, pb, tune);
     if (!pl.ok) return cudaErrorNotSupported;
     TcParams prm{};
     prm.lr = lr; prm.dict = dict; prm.out = out; prm.idx = idx; prm.gamma = gamma;

@@ -299,15 +299,6 @@ select_scan_kernel(const CoefT* __restrict__ coef, uint8_t* __restrict__ idx, Co
     }
 }
 
-int sm_count()
-{
-    static int sms[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms[dev] = 148;
-    return sms[dev];
-}
-
 template <typename CoefT>
 cudaError_t launch_sel(const void* coef, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
 {
