@@ -14,7 +14,7 @@
  *     as void* (NULL = the legacy default stream).  `d` is a HOST pointer.
  *   - Layouts, all contiguous, row-major, innermost index last:
  *       lr        [n][c][h][w]           fp32   LR image
- *       hr / out  [n][c][H][W]           fp32   H = h*scale, W = w*scale (out: binary16 with SR_OUT_F16)
+ *       hr / out  [n][c][H][W]           fp32   H = h*scale, W = w*scale (out: binary16 with SR_OUT_F16, uint8 with SR_OUT_U8)
  *       coef      [n][D][H][W]           fp32 or binary16 (SR_F32 / SR_F16); one set per
  *                                        frame, shared by the c channels
  *       dict      [D][k*k]               fp32, tap j = a*k + b (a = row) multiplies
@@ -72,8 +72,12 @@ enum {
     SR_COEF_COMPACT = 4u, /* the coefficient argument is [n][s][H][W] (selected values), not [n][D][H][W] */
     SR_UPSAMPLE_BILINEAR = 8u, /* stage 1 interpolates linearly between the two nearest LR samples per axis
                                   (the interpolation Section II-A names) instead of the bicubic kernel        */
-    SR_OUT_F16 = 16u           /* regression calls: `out` is binary16 [n][c][H][W]; the fp32 result is rounded
+    SR_OUT_F16 = 16u,          /* regression calls: `out` is binary16 [n][c][H][W]; the fp32 result is rounded
                                   to nearest as it is stored (halves the output traffic).  2-byte alignment.  */
+    SR_OUT_U8 = 32u            /* regression calls: `out` is uint8 [n][c][H][W], an 8-bit image: the fp32 result
+                                  clamped to [0,1] (whether or not SR_CLAMP01 is given), times 255, rounded to
+                                  nearest, ties to even (a quarter of the output traffic).  Not together with
+                                  SR_OUT_F16.                                                                  */
 };
 
 enum {

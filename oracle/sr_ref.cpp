@@ -44,7 +44,7 @@
 namespace {
 
 enum { REF_F32 = 0, REF_F16 = 1 };
-enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u, REF_UPSAMPLE_BILINEAR = 8u };
+enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u, REF_UPSAMPLE_BILINEAR = 8u, REF_OUT_U8 = 32u };
 enum { REF_OK = 0, REF_ERR_NULL = 1, REF_ERR_SHAPE = 2, REF_ERR_UNSUPPORTED = 3 };
 
 struct Dims {
@@ -173,6 +173,12 @@ void regress_pixel(const Dims& d, const float* dict, int natoms, const int* atom
                 acc += F[a * k + b] * patch(ch, yy, xx);
             }
         if (flags & REF_CLAMP01) acc = acc < 0.0 ? 0.0 : (acc > 1.0 ? 1.0 : acc);
+        if (flags & REF_OUT_U8) {
+            /* 8-bit image output (an I/O variant of this build, not in the paper): the code of the value clamped to
+             * [0,1] on the 255-step grid, nearest code, ties to the even one */
+            const double v = acc < 0.0 ? 0.0 : (acc > 1.0 ? 1.0 : acc);
+            acc = std::nearbyint(255.0 * v);
+        }
         y[ch] = acc;
     }
 }

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsr.so")
 
 SR_F32, SR_F16 = 0, 1
-SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16 = 1, 2, 4, 8, 16
+SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16, SR_OUT_U8 = 1, 2, 4, 8, 16, 32
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT, SR_ERR_TOO_LARGE = range(8)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
@@ -116,6 +116,10 @@ def _coef_code(t: torch.Tensor) -> int:
     raise TypeError("coefficients must be float16 or float32")
 
 
+def _out_dtype(flags: int):
+    return torch.uint8 if (flags & SR_OUT_U8) else (torch.float16 if (flags & SR_OUT_F16) else torch.float32)
+
+
 def _check(status: int, what: str):
     if status != SR_OK:
         raise SrError(status, what)
@@ -148,7 +152,7 @@ def sr_dict_regress_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, o
     n, c, h, w = lr.shape
     D = dict_.shape[0]
     assert dict_.shape == (D, k * k) and coef.shape == (n, D, h * scale, w * scale)
-    out_dtype = torch.float16 if (flags & SR_OUT_F16) else torch.float32
+    out_dtype = _out_dtype(flags)
     if out is None:
         out = torch.empty((n, c, h * scale, w * scale), dtype=out_dtype, device=lr.device)
     _dev(out, out_dtype, "out")
@@ -190,7 +194,7 @@ def sr_dict_regress_selected(lr, coef_or_sel, idx, gamma, dict_, scale: int, k: 
     assert dict_.shape == (D, k * k)
     planes = s if (flags & SR_COEF_COMPACT) else D
     assert coef_or_sel.shape == (n, planes, h * scale, w * scale)
-    out_dtype = torch.float16 if (flags & SR_OUT_F16) else torch.float32
+    out_dtype = _out_dtype(flags)
     if out is None:
         out = torch.empty((n, c, h * scale, w * scale), dtype=out_dtype, device=lr.device)
     _dev(out, out_dtype, "out")
@@ -296,7 +300,7 @@ def sr_tune_dense(lr, coef, dict_, scale: int, k: int, flags: int = 0, reps: int
     code = _coef_code(coef)
     n, c, h, w = lr.shape
     D = dict_.shape[0]
-    out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float16 if (flags & SR_OUT_F16) else torch.float32, device=lr.device)
+    out = torch.empty((n, c, h * scale, w * scale), dtype=_out_dtype(flags), device=lr.device)
     d = sr_dims(n, c, h, w, scale, k, D)
     res = sr_tune_result()
     _check(load_library().sr_tune_dense(_ptr(lr), _ptr(coef), code, _ptr(dict_), _ptr(out), ctypes.byref(d), flags, reps, _stream(),
@@ -310,7 +314,7 @@ def sr_tune_selected(lr, coef_or_sel, idx, gamma, dict_, scale: int, k: int, s: 
     code = _coef_code(coef_or_sel)
     n, c, h, w = lr.shape
     D = dict_.shape[0]
-    out = torch.empty((n, c, h * scale, w * scale), dtype=torch.float16 if (flags & SR_OUT_F16) else torch.float32, device=lr.device)
+    out = torch.empty((n, c, h * scale, w * scale), dtype=_out_dtype(flags), device=lr.device)
     d = sr_dims(n, c, h, w, scale, k, D)
     res = sr_tune_result()
     _check(load_library().sr_tune_selected(_ptr(lr), _ptr(coef_or_sel), code, _ptr(idx), _ptr(gamma), _ptr(dict_), _ptr(out),

@@ -110,6 +110,8 @@ static Problem make_problem(const sr_dims* d, int s, uint32_t flags)
 }
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+static size_t out_align(uint32_t flags) { return (flags & SR_OUT_U8) ? 1 : ((flags & SR_OUT_F16) ? 2 : 4); }
+static bool bad_out_flags(uint32_t flags) { return (flags & SR_OUT_F16) && (flags & SR_OUT_U8); }   // one output type at a time
 
 // Which tensor-core layout takes a dense launch. The second layout (sr_regress_tc.cu: channel-split epilogue, two CTAs
 // per SM, several rows per pipeline step) wins where the coefficient stream is light and the epilogue sets the pace:
@@ -306,8 +308,8 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
     return run_regress(a) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
@@ -319,8 +321,8 @@ int sr_tune_dense(const float* lr, const void* coef, int coef_dtype, const float
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
     return tune_shape(a, reps, result);
@@ -349,11 +351,11 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
+    if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
         !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{selected_mode(idx, flags), lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, make_problem(d, s, flags), (cudaStream_t)stream};
@@ -367,11 +369,11 @@ int sr_tune_selected(const float* lr, const void* coef_or_sel, int coef_dtype, c
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
-    if (!aligned(lr, 4) || !aligned(out, (flags & SR_OUT_F16) ? 2 : 4) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
+    if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || (gamma && !aligned(gamma, 4)) ||
         !aligned(coef_or_sel, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{selected_mode(idx, flags), lr, coef_or_sel, coef_dtype, idx, gamma, dict, out, make_problem(d, s, flags), (cudaStream_t)stream};

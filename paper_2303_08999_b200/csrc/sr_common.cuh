@@ -71,12 +71,15 @@ __device__ __forceinline__ int clampi(int v, int lo, int hi) { return min(max(v,
 template <typename OutT> __device__ __forceinline__ OutT to_out(float v);
 template <> __device__ __forceinline__ float to_out<float>(float v) { return v; }
 template <> __device__ __forceinline__ __half to_out<__half>(float v) { return __float2half_rn(v); }
+// SR_OUT_U8: the value clamped to [0, 1], times 255, rounded to nearest (ties to even)
+template <> __device__ __forceinline__ uint8_t to_out<uint8_t>(float v) { return (uint8_t)__float2int_rn(fminf(fmaxf(v, 0.f), 1.f) * 255.f); }
 
 // Output element i of a frame buffer that holds fp32 or (f16) binary16 values; for kernels that are not tight on
 // registers and take the output type at run time.
-__device__ __forceinline__ void store_out(float* out, int64_t i, float v, bool f16)
+__device__ __forceinline__ void store_out(float* out, int64_t i, float v, uint32_t flags)
 {
-    if (f16) reinterpret_cast<__half*>(out)[i] = __float2half_rn(v);
+    if (flags & SR_OUT_U8) reinterpret_cast<uint8_t*>(out)[i] = to_out<uint8_t>(v);
+    else if (flags & SR_OUT_F16) reinterpret_cast<__half*>(out)[i] = __float2half_rn(v);
     else out[i] = v;
 }
 

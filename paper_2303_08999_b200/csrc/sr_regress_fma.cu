@@ -116,7 +116,7 @@ regress_fma_kernel(const float* __restrict__ lr, const CoefT* __restrict__ coef,
 #pragma unroll
                 for (int b = 0; b < K; ++b) acc = fmaf(F[a * K + b], u[a * UW + b], acc);
             if (pb.flags & SR_CLAMP01) acc = fminf(fmaxf(acc, 0.f), 1.f);
-            if (valid) store_out(out, ((int64_t)f * pb.c + c0 + ch) * HW + pix, acc, (pb.flags & SR_OUT_F16) != 0);
+            if (valid) store_out(out, ((int64_t)f * pb.c + c0 + ch) * HW + pix, acc, pb.flags);
         }
     }
 }

@@ -195,6 +195,8 @@ __global__ void __launch_bounds__(kThreads, 2) regress_subset_kernel(const __gri
                     OutT* o = of + c * plane_elems + pix;
                     if constexpr (sizeof(OutT) == 4) {
                         *reinterpret_cast<float4*>(o) = make_float4(v[0], v[1], v[2], v[3]);
+                    } else if constexpr (sizeof(OutT) == 1) {
+                        *reinterpret_cast<uchar4*>(o) = make_uchar4(to_out<uint8_t>(v[0]), to_out<uint8_t>(v[1]), to_out<uint8_t>(v[2]), to_out<uint8_t>(v[3]));
                     } else {
                         const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
                         *reinterpret_cast<uint2*>(o) = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
@@ -278,6 +280,7 @@ cudaError_t launch_t(const SubParams& prm, int ctas, size_t smem, cudaStream_t s
 template <int K, int NQ, int C>
 cudaError_t launch_o(const SubParams& prm, int ctas, size_t smem, cudaStream_t st)
 {
+    if (prm.g.pb.flags & SR_OUT_U8) return launch_t<K, NQ, C, uint8_t>(prm, ctas, smem, st);
     if (prm.g.pb.flags & SR_OUT_F16) return launch_t<K, NQ, C, __half>(prm, ctas, smem, st);
     return launch_t<K, NQ, C, float>(prm, ctas, smem, st);
 }
@@ -312,7 +315,7 @@ int regress_subset_candidates(const Problem& pb, int* ths, int max_out)
 
 bool regress_subset_supported(int mode, const void* coef, int coef_dtype, const void* out, const Problem& pb)
 {
-    if ((reinterpret_cast<uintptr_t>(out) & ((pb.flags & SR_OUT_F16) ? 7 : 15)) != 0) return false;            // one store per four pixels
+    if ((reinterpret_cast<uintptr_t>(out) & ((pb.flags & SR_OUT_U8) ? 3 : ((pb.flags & SR_OUT_F16) ? 7 : 15))) != 0) return false;   // one store per four pixels
     if (mode != kModeGlobal || pb.s > 8 || coef_dtype != SR_F16) return false;
     if (pb.k > 7 || (pb.c != 1 && pb.c != 3)) return false;
     if ((reinterpret_cast<uintptr_t>(coef) & 7) != 0 || (pb.W & 3) != 0) return false;    // 8-byte loads of four coefficients

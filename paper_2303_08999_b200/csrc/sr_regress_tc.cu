@@ -700,6 +700,7 @@ cudaError_t launch_kho(const CUtensorMap& map_lead, const TcParams& prm, const P
 template <int K, bool HILO>
 cudaError_t launch_kh(const CUtensorMap& map_lead, const TcParams& prm, const Plan& pl, cudaStream_t st)
 {
+    if (prm.g.pb.flags & SR_OUT_U8) return launch_kho<K, HILO, uint8_t>(map_lead, prm, pl, st);
     if (prm.g.pb.flags & SR_OUT_F16) return launch_kho<K, HILO, __half>(map_lead, prm, pl, st);
     return launch_kho<K, HILO, float>(map_lead, prm, pl, st);
 }

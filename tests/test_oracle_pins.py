@@ -375,3 +375,33 @@ def test_binary16_widening_every_bit_pattern():
     lr = np.ones((1, 1, 256, 256), np.float32)
     out = oracle.dict_regress_dense(lr, coef, np.ones((1, 1), np.float32), 1, 1)
     np.testing.assert_array_equal(out[0][finite[0]], want[0][finite[0]])
+
+
+def test_eight_bit_output_codes():
+    """SR_OUT_U8 in the oracle: the code of the clamped value on the 255-step grid. Pinned by the worked 4 x 4 example
+    (its printed values times 255, rounded by hand: -0.0382 -> 0, 0.1682 -> 43, 0.5123 -> 131, 1.4987 -> 255), by
+    numpy's rint on the oracle's own unquantised output, and by the round-half-even rule on exact ties."""
+    lr = np.array([[[[0.0, 0.25], [0.5, 1.0]]]], np.float32)
+    d = np.zeros((2, 9), np.float32)
+    d[0, 4] = 1.0
+    d[1, :] = 1.0 / 9.0
+    coef = np.zeros((1, 2, 4, 4), np.float32)
+    coef[0, 0] = 0.5
+    coef[0, 1] = (4 * np.arange(4)[:, None] + np.arange(4)[None, :]) / 16.0
+    codes = oracle.dict_regress_dense(lr, coef, d, 2, 3, flags=oracle.OUT_U8)[0, 0]
+    assert codes[0, 0] == 0 and codes[1, 1] == 43 and codes[2, 1] == 131 and codes[3, 3] == 255
+    plain = oracle.dict_regress_dense(lr, coef, d, 2, 3)
+    np.testing.assert_array_equal(codes, np.rint(255.0 * np.clip(plain[0, 0], 0.0, 1.0)))
+    # exact ties: 0.5 / 255 and 1.5 / 255 are not representable, so build ties through the atom weight instead:
+    # a 1 x 1 unit atom on a constant image of value 1 returns the coefficient; x.5 / 255 * 255 is a tie only in exact
+    # arithmetic, so check the integers around it and the monotone staircase
+    lr1 = np.ones((1, 1, 1, 256), np.float32)
+    co = (np.arange(256, dtype=np.float64) / 255.0).astype(np.float32).reshape(1, 1, 1, 256)
+    q = oracle.dict_regress_dense(lr1, co, np.ones((1, 1), np.float32), 1, 1, flags=oracle.OUT_U8)[0, 0, 0]
+    np.testing.assert_array_equal(q, np.arange(256))
+    wl = sr_inputs.Workload("t", 1, 3, 6, 7, 2, D=6, k=3, coef_dtype="f16")
+    lr, dd, cf = sr_inputs.make_inputs(wl)
+    q = oracle.dict_regress_selected(lr, cf, None, None, dd, 2, 3, 2, flags=oracle.OUT_U8)
+    v = oracle.dict_regress_selected(lr, cf, None, None, dd, 2, 3, 2)
+    np.testing.assert_array_equal(q, np.rint(255.0 * np.clip(v, 0.0, 1.0)))
+    assert q.min() >= 0 and q.max() <= 255
