@@ -72,7 +72,8 @@ def test_validation_errors_come_back_before_any_launch(lib):
     # the up-sampling variant is a legal flag of the regression calls: validation goes on to the next check
     assert dense(_dims(k=4), flags=api.SR_UPSAMPLE_BILINEAR) == api.SR_ERR_UNSUPPORTED
     assert dense(_dims(), flags=api.SR_UPSAMPLE_BILINEAR | api.SR_CLAMP01, coef=FAKE + 1) == api.SR_ERR_ALIGN
-    assert dense(_dims(), flags=32) == api.SR_ERR_UNSUPPORTED
+    assert dense(_dims(), flags=64) == api.SR_ERR_UNSUPPORTED                      # an unknown flag
+    assert dense(_dims(), flags=api.SR_OUT_F16 | api.SR_OUT_U8) == api.SR_ERR_UNSUPPORTED   # one output type at a time
     # binary16 output: `out` needs 2-byte alignment only (FAKE + 2 passes this check and fails the next one)
     out_at = lambda out, flags: lib.sr_dict_regress_dense(FAKE, FAKE + 1, api.SR_F16, FAKE, out, ctypes.byref(_dims()), flags, None)
     assert lib.sr_dict_regress_dense(FAKE, FAKE, api.SR_F16, FAKE, FAKE + 2, ctypes.byref(_dims()), 0, None) == api.SR_ERR_ALIGN
