@@ -74,10 +74,15 @@ enum {
                                   (the interpolation Section II-A names) instead of the bicubic kernel        */
     SR_OUT_F16 = 16u,          /* regression calls: `out` is binary16 [n][c][H][W]; the fp32 result is rounded
                                   to nearest as it is stored (halves the output traffic).  2-byte alignment.  */
-    SR_OUT_U8 = 32u            /* regression calls: `out` is uint8 [n][c][H][W], an 8-bit image: the fp32 result
+    SR_OUT_U8 = 32u,           /* regression calls: `out` is uint8 [n][c][H][W], an 8-bit image: the fp32 result
                                   clamped to [0,1] (whether or not SR_CLAMP01 is given), times 255, rounded to
                                   nearest, ties to even (a quarter of the output traffic).  Not together with
                                   SR_OUT_F16.                                                                  */
+    SR_LUMA_ONLY = 64u         /* regression calls, c = 3 (R, G, B planes) only: the per-pixel filter is applied to
+                                  the luma Y = 0.299 R + 0.587 G + 0.114 B of the up-sampled image and the chroma
+                                  differences keep their up-sampled values:  out_ch = U_ch + (F . B_Y - U_Y)  at the
+                                  pixel.  The common practice of SR models that predict on the Y channel; the paper
+                                  has no such variant.  Runs on the general fp32 kernel, whatever the shape.   */
 };
 
 enum {

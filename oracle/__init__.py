@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "sr_ref.cpp")
 _LIB = os.path.join(_HERE, "libsr_ref.so")
 
 F32, F16 = 0, 1
-CLAMP01, IDX_GLOBAL, COEF_COMPACT, UPSAMPLE_BILINEAR, OUT_U8 = 1, 2, 4, 8, 32
+CLAMP01, IDX_GLOBAL, COEF_COMPACT, UPSAMPLE_BILINEAR, OUT_U8, LUMA_ONLY = 1, 2, 4, 8, 32, 64
 
 _lib = None
 

@@ -44,7 +44,7 @@
 namespace {
 
 enum { REF_F32 = 0, REF_F16 = 1 };
-enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u, REF_UPSAMPLE_BILINEAR = 8u, REF_OUT_U8 = 32u };
+enum { REF_CLAMP01 = 1u, REF_IDX_GLOBAL = 2u, REF_COEF_COMPACT = 4u, REF_UPSAMPLE_BILINEAR = 8u, REF_OUT_U8 = 32u, REF_LUMA_ONLY = 64u };
 enum { REF_OK = 0, REF_ERR_NULL = 1, REF_ERR_SHAPE = 2, REF_ERR_UNSUPPORTED = 3 };
 
 struct Dims {
@@ -164,14 +164,36 @@ void regress_pixel(const Dims& d, const float* dict, int natoms, const int* atom
     for (int j = 0; j < kk; ++j) F[j] = 0.0;
     for (int q = 0; q < natoms; ++q)
         for (int j = 0; j < kk; ++j) F[j] += weights[q] * (double)dict[(int64_t)atoms[q] * kk + j];
-    for (int ch = 0; ch < d.c; ++ch) {
+    /*
+     * Luma-only regression (an I/O variant of this build, the usual practice of SR models that work on the Y channel;
+     * not in the paper): the filter is applied to the luma Y = 0.299 R + 0.587 G + 0.114 B (BT.601) of the up-sampled
+     * image, the two chroma differences keep their up-sampled values.  In RGB that is
+     *     out_c = U_c + (F . B_Y - U_Y)       at the pixel, for c = R, G, B  (needs c = 3).
+     */
+    double luma_shift = 0.0;
+    if (flags & REF_LUMA_ONLY) {
+        const double wy[3] = {0.299, 0.587, 0.114};
         double acc = 0.0;
         for (int a = 0; a < k; ++a)
             for (int b = 0; b < k; ++b) {
                 const int yy = clampi(Y + a - p, 0, d.H() - 1);
                 const int xx = clampi(X + b - p, 0, d.W() - 1);
-                acc += F[a * k + b] * patch(ch, yy, xx);
+                acc += F[a * k + b] * (wy[0] * patch(0, yy, xx) + wy[1] * patch(1, yy, xx) + wy[2] * patch(2, yy, xx));
             }
+        luma_shift = acc - (wy[0] * patch(0, Y, X) + wy[1] * patch(1, Y, X) + wy[2] * patch(2, Y, X));
+    }
+    for (int ch = 0; ch < d.c; ++ch) {
+        double acc = 0.0;
+        if (flags & REF_LUMA_ONLY) {
+            acc = patch(ch, Y, X) + luma_shift;
+        } else {
+            for (int a = 0; a < k; ++a)
+                for (int b = 0; b < k; ++b) {
+                    const int yy = clampi(Y + a - p, 0, d.H() - 1);
+                    const int xx = clampi(X + b - p, 0, d.W() - 1);
+                    acc += F[a * k + b] * patch(ch, yy, xx);
+                }
+        }
         if (flags & REF_CLAMP01) acc = acc < 0.0 ? 0.0 : (acc > 1.0 ? 1.0 : acc);
         if (flags & REF_OUT_U8) {
             /* 8-bit image output (an I/O variant of this build, not in the paper): the code of the value clamped to
@@ -435,6 +457,7 @@ int sr_ref_dict_regress_dense(const float* lr, const void* coef, int coef_dtype,
     Dims d{n, c, h, w, r, k, L};
     if (!lr || !coef || !dict || !out) return REF_ERR_NULL;
     if (int e = check_dims(d)) return e;
+    if ((flags & REF_LUMA_ONLY) && c != 3) return REF_ERR_UNSUPPORTED;
     set_threads(threads);
     const int H = d.H(), W = d.W();
     const int64_t HW = (int64_t)H * W;
@@ -500,6 +523,7 @@ int sr_ref_dict_regress_selected(const float* lr, const void* coef_or_sel, int c
     if (!lr || !coef_or_sel || !dict || !out) return REF_ERR_NULL;
     if ((flags & (REF_IDX_GLOBAL | REF_COEF_COMPACT)) && !idx) return REF_ERR_NULL;
     if (int e = check_dims(d)) return e;
+    if ((flags & REF_LUMA_ONLY) && c != 3) return REF_ERR_UNSUPPORTED;
     if (s < 1 || s > L) return REF_ERR_SHAPE;
     if (flags & REF_IDX_GLOBAL)
         for (int q = 0; q < s; ++q)
@@ -539,6 +563,7 @@ int sr_ref_regress_at(int mode, const float* lr, const void* coef_or_sel, int co
     Dims d{n, c, h, w, r, k, L};
     if (!lr || !coef_or_sel || !dict || !out || !samples) return REF_ERR_NULL;
     if (int e = check_dims(d)) return e;
+    if ((flags & REF_LUMA_ONLY) && c != 3) return REF_ERR_UNSUPPORTED;
     if (mode == 0) s = L;
     if (s < 1 || s > L) return REF_ERR_SHAPE;
     if (mode == 1 && (flags & (REF_IDX_GLOBAL | REF_COEF_COMPACT)) && !idx) return REF_ERR_NULL;

@@ -111,7 +111,11 @@ static Problem make_problem(const sr_dims* d, int s, uint32_t flags)
 
 static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 static size_t out_align(uint32_t flags) { return (flags & SR_OUT_U8) ? 1 : ((flags & SR_OUT_F16) ? 2 : 4); }
-static bool bad_out_flags(uint32_t flags) { return (flags & SR_OUT_F16) && (flags & SR_OUT_U8); }   // one output type at a time
+// one output type at a time; luma-only regression needs the three colour planes
+static bool bad_out_flags(uint32_t flags, const sr_dims* d)
+{
+    return ((flags & SR_OUT_F16) && (flags & SR_OUT_U8)) || ((flags & SR_LUMA_ONLY) && d->c != 3);
+}
 
 // Which tensor-core layout takes a dense launch. The second layout (sr_regress_tc.cu: channel-split epilogue, two CTAs
 // per SM, several rows per pipeline step) wins where the coefficient stream is light and the epilogue sets the pace:
@@ -176,6 +180,7 @@ struct RegressArgs {
 static bool kernel_supported(int kernel, const RegressArgs& a)
 {
     const bool idx_vec_ok = !a.idx || a.mode == kModeGlobal || ((reinterpret_cast<uintptr_t>(a.idx) & 15) == 0);   // 16-byte reads
+    if ((a.pb.flags & SR_LUMA_ONLY) && kernel != kKernelGeneral) return false;   // only the general kernel has the luma variant
     switch (kernel) {
     case kKernelSubset: return regress_subset_supported(a.mode, a.coef, a.coef_dtype, a.out, a.pb);
     case kKernelSecondLayout: return regress_tc_supported(a.mode, a.coef, a.coef_dtype, a.pb);
@@ -308,7 +313,7 @@ int sr_dict_regress_dense(const float* lr, const void* coef, int coef_dtype, con
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8 | SR_LUMA_ONLY) || bad_out_flags(flags, d)) return SR_ERR_UNSUPPORTED;
     if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
@@ -321,7 +326,7 @@ int sr_tune_dense(const float* lr, const void* coef, int coef_dtype, const float
     if (!lr || !coef || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8 | SR_LUMA_ONLY) || bad_out_flags(flags, d)) return SR_ERR_UNSUPPORTED;
     if (!aligned(lr, 4) || !aligned(out, out_align(flags)) || !aligned(dict, 4) || !aligned(coef, coef_dtype == SR_F16 ? 2 : 4))
         return SR_ERR_ALIGN;
     const RegressArgs a{kModeDense, lr, coef, coef_dtype, nullptr, nullptr, dict, out, make_problem(d, d->D, flags), (cudaStream_t)stream};
@@ -351,7 +356,7 @@ int sr_dict_regress_selected(const float* lr, const void* coef_or_sel, int coef_
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8 | SR_LUMA_ONLY) || bad_out_flags(flags, d)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;
@@ -369,7 +374,7 @@ int sr_tune_selected(const float* lr, const void* coef_or_sel, int coef_dtype, c
     if (!lr || !coef_or_sel || !dict || !out || !d) return SR_ERR_NULL;
     if (int e = check_dims(d, true)) return e;
     if (coef_dtype != SR_F32 && coef_dtype != SR_F16) return SR_ERR_UNSUPPORTED;
-    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags)) return SR_ERR_UNSUPPORTED;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_IDX_GLOBAL | SR_COEF_COMPACT | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8 | SR_LUMA_ONLY) || bad_out_flags(flags, d)) return SR_ERR_UNSUPPORTED;
     if (s < 1 || s > d->D) return SR_ERR_SHAPE;
     if ((flags & (SR_IDX_GLOBAL | SR_COEF_COMPACT)) && !idx) return SR_ERR_NULL;
     if (gamma && !(flags & SR_IDX_GLOBAL)) return SR_ERR_UNSUPPORTED;

@@ -108,6 +108,27 @@ regress_fma_kernel(const float* __restrict__ lr, const CoefT* __restrict__ coef,
             sU[i] = bicubic_point(plane, pb.h, pb.w, pb.r, pb.ph, clampi(Y0 + uy, 0, H - 1), clampi(X0 + ux, 0, W - 1));
         }
         __syncthreads();
+        if (pb.flags & SR_LUMA_ONLY) {
+            // c = 3 (checked by the caller): the fourth slot takes the luma of the tile, the filter runs on it once,
+            // and every channel moves by the same amount, so the chroma differences stay those of stage 1.
+            float* sY = sU + 3 * UH * UW;
+            for (int i = tid; i < UH * UW; i += TX * TY)
+                sY[i] = fmaf(0.299f, sU[i], fmaf(0.587f, sU[UH * UW + i], 0.114f * sU[2 * UH * UW + i]));
+            __syncthreads();
+            const float* u = sY + threadIdx.y * UW + threadIdx.x;
+            float acc = 0.f;
+#pragma unroll
+            for (int a = 0; a < K; ++a)
+#pragma unroll
+                for (int b = 0; b < K; ++b) acc = fmaf(F[a * K + b], u[a * UW + b], acc);
+            const float shift = acc - u[P * UW + P];
+            for (int ch = 0; ch < 3; ++ch) {
+                float v = sU[ch * UH * UW + (threadIdx.y + P) * UW + threadIdx.x + P] + shift;
+                if (pb.flags & SR_CLAMP01) v = fminf(fmaxf(v, 0.f), 1.f);
+                if (valid) store_out(out, ((int64_t)f * 3 + ch) * HW + pix, v, pb.flags);
+            }
+            break;
+        }
         for (int ch = 0; ch < nc; ++ch) {
             const float* u = sU + ch * UH * UW + threadIdx.y * UW + threadIdx.x;
             float acc = 0.f;

@@ -72,7 +72,9 @@ def test_validation_errors_come_back_before_any_launch(lib):
     # the up-sampling variant is a legal flag of the regression calls: validation goes on to the next check
     assert dense(_dims(k=4), flags=api.SR_UPSAMPLE_BILINEAR) == api.SR_ERR_UNSUPPORTED
     assert dense(_dims(), flags=api.SR_UPSAMPLE_BILINEAR | api.SR_CLAMP01, coef=FAKE + 1) == api.SR_ERR_ALIGN
-    assert dense(_dims(), flags=64) == api.SR_ERR_UNSUPPORTED                      # an unknown flag
+    assert dense(_dims(), flags=128) == api.SR_ERR_UNSUPPORTED                     # an unknown flag
+    assert dense(_dims(c=1), flags=api.SR_LUMA_ONLY) == api.SR_ERR_UNSUPPORTED     # luma-only needs R, G, B planes
+    assert dense(_dims(c=3), flags=api.SR_LUMA_ONLY, coef=FAKE + 1) == api.SR_ERR_ALIGN   # legal with c = 3: next check
     assert dense(_dims(), flags=api.SR_OUT_F16 | api.SR_OUT_U8) == api.SR_ERR_UNSUPPORTED   # one output type at a time
     # binary16 output: `out` needs 2-byte alignment only (FAKE + 2 passes this check and fails the next one)
     out_at = lambda out, flags: lib.sr_dict_regress_dense(FAKE, FAKE + 1, api.SR_F16, FAKE, out, ctypes.byref(_dims()), flags, None)
@@ -92,7 +94,8 @@ def test_validation_errors_come_back_before_any_launch(lib):
     assert selected(_dims(), 4, flags=api.SR_IDX_GLOBAL, idx=None) == api.SR_ERR_NULL
     assert selected(_dims(), 4, flags=api.SR_COEF_COMPACT, idx=None) == api.SR_ERR_NULL
     assert selected(_dims(), 4, gamma=FAKE) == api.SR_ERR_UNSUPPORTED  # gamma only exists for the global subset
-    assert selected(_dims(), 4, flags=64) == api.SR_ERR_UNSUPPORTED
+    assert selected(_dims(), 4, flags=128) == api.SR_ERR_UNSUPPORTED
+    assert selected(_dims(c=1), 4, flags=api.SR_LUMA_ONLY) == api.SR_ERR_UNSUPPORTED
     assert lib.sr_device_status(None, None) == api.SR_ERR_NULL
 
 

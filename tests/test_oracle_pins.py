@@ -405,3 +405,40 @@ def test_eight_bit_output_codes():
     v = oracle.dict_regress_selected(lr, cf, None, None, dd, 2, 3, 2)
     np.testing.assert_array_equal(q, np.rint(255.0 * np.clip(v, 0.0, 1.0)))
     assert q.min() >= 0 and q.max() <= 255
+
+
+def test_luma_only_regression():
+    """LUMA_ONLY in the oracle (filter the BT.601 luma of the up-sampled image, keep the up-sampled chroma), pinned by:
+    the composition out = U + (regression of the luma image - luma of U) built from the pinned one-channel regression
+    and bicubic (stage 1 is linear, so up-sampling the luma of the LR image is the luma of the up-sampled image);
+    chroma differences that equal those of U; a grey image, where it is the ordinary regression; the delta atom."""
+    wy = np.array([0.299, 0.587, 0.114])
+    wl = sr_inputs.Workload("t", 2, 3, 7, 9, 3, D=6, k=5, coef_dtype="f16")
+    lr, d, coef = sr_inputs.make_inputs(wl)
+    d = (d + np.random.default_rng(1).normal(0, 0.1, d.shape)).astype(np.float32)
+    out = oracle.dict_regress_dense(lr, coef, d, 3, 5, flags=oracle.LUMA_ONLY)
+    U = oracle.bicubic_upsample(lr, 3)
+    UY = np.tensordot(wy, U, axes=([0], [1]))[:, None]                       # [n][1][H][W]
+    lrY = np.tensordot(wy, lr.astype(np.float64), axes=([0], [1]))[:, None]
+    regY = oracle.dict_regress_dense(lrY.astype(np.float32), coef, d, 3, 5)  # the luma image through the one-channel path
+    want = U + (regY - UY)
+    assert np.abs(out - want).max() <= 5e-7                                  # fp32 rounding of the luma LR image only
+    outY = np.tensordot(wy, out, axes=([0], [1]))[:, None]
+    assert np.abs((out - outY) - (U - UY)).max() <= 1e-12                    # chroma differences untouched
+    # selected modes go through the same pixel routine
+    sel = oracle.dict_regress_selected(lr, coef, None, None, d, 3, 5, 2, flags=oracle.LUMA_ONLY)
+    regY = oracle.dict_regress_selected(lrY.astype(np.float32), coef, None, None, d, 3, 5, 2)
+    assert np.abs(sel - (U + (regY - UY))).max() <= 5e-7
+    # grey image: luma = every channel, so nothing changes
+    grey = np.repeat(lr[:, :1], 3, axis=1)
+    a = oracle.dict_regress_dense(grey, coef, d, 3, 5, flags=oracle.LUMA_ONLY)
+    b = oracle.dict_regress_dense(grey, coef, d, 3, 5)
+    assert np.abs(a - b).max() <= 1e-12
+    # delta atom, one-hot coefficients: the up-sampled image itself
+    dd = np.zeros_like(d)
+    dd[0, 12] = 1.0
+    one = np.zeros_like(coef)
+    one[:, 0] = 1.0
+    assert np.abs(oracle.dict_regress_dense(lr, one, dd, 3, 5, flags=oracle.LUMA_ONLY) - U).max() <= 1e-12
+    with pytest.raises(ValueError):
+        oracle.dict_regress_dense(lr[:, :2], coef, d, 3, 5, flags=oracle.LUMA_ONLY)
