@@ -48,6 +48,8 @@ def _load():
         L.sr_ref_selection_search.argtypes = [vp, vp, f64, i32, f64, f64, f64, f64, f64, f64, i32, i32, vp, vp, vp, vp, i32, vp]
         for f in (L.sr_ref_selection_gram, L.sr_ref_lasso_cd, L.sr_ref_selection_search):
             f.restype = i32
+        L.sr_ref_producer_coef.argtypes = [vp, vp, vp, vp] + [i32] * 8
+        L.sr_ref_producer_regress.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp] + [i32] * 9 + [u32, i32]
         L.sr_ref_max_threads.argtypes = []
         for f in (L.sr_ref_bicubic_upsample, L.sr_ref_bilinear_upsample, L.sr_ref_dict_regress_dense, L.sr_ref_dict_select,
                   L.sr_ref_dict_regress_selected, L.sr_ref_regress_at, L.sr_ref_dict_select_at, L.sr_ref_max_threads):
@@ -202,3 +204,41 @@ def selection_search(G, b, hh: float, nrows: float, alpha: float, delta_alpha: f
                                            gamma.ctypes.data, ctypes.addressof(count), trace.ctypes.data, max_steps,
                                            ctypes.addressof(steps)), "selection_search")
     return idx[: count.value].copy(), gamma[: count.value].copy(), trace[: steps.value].copy()
+
+
+def producer_coef(feat, wconv, bias, scale: int, threads: int = 0) -> np.ndarray:
+    """Phi [n][L][H][W] (fp64) from the LR feature map feat [n][h][w][cin] (float16), the last convolution
+    wconv [L r^2][cin][kc][kc] (+ bias [L r^2] or None) and the pixel-shuffle by `scale`."""
+    feat, wconv = _c(feat, np.float16), _c(wconv, np.float32)
+    n, h, w, cin = feat.shape
+    cout, cin2, kc, kc2 = wconv.shape
+    assert cin2 == cin and kc2 == kc and cout % (scale * scale) == 0
+    L = cout // (scale * scale)
+    bias = None if bias is None else _c(bias, np.float32)
+    assert bias is None or bias.shape == (cout,)
+    phi = np.empty((n, L, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_producer_coef(feat.ctypes.data, wconv.ctypes.data, None if bias is None else bias.ctypes.data,
+                                        phi.ctypes.data, n, h, w, scale, L, cin, kc, threads), "producer_coef")
+    return phi
+
+
+def producer_regress(lr, feat, wconv, bias, dict_, scale: int, k: int, idx=None, gamma=None, flags: int = 0,
+                     threads: int = 0) -> np.ndarray:
+    """The dense regression (or the global-subset one, with idx / gamma) with Phi computed from the feature map."""
+    lr, feat, wconv, dict_ = _c(lr, np.float32), _c(feat, np.float16), _c(wconv, np.float32), _c(dict_, np.float32)
+    n, c, h, w = lr.shape
+    assert feat.shape[:3] == (n, h, w)
+    cin = feat.shape[3]
+    cout, cin2, kc, kc2 = wconv.shape
+    D = dict_.shape[0]
+    assert cin2 == cin and kc2 == kc and cout == D * scale * scale and dict_.shape == (D, k * k)
+    bias = None if bias is None else _c(bias, np.float32)
+    idx = None if idx is None else _c(idx, np.uint8)
+    gamma = None if gamma is None else _c(gamma, np.float32)
+    s = 0 if idx is None else idx.size
+    out = np.empty((n, c, h * scale, w * scale), dtype=np.float64)
+    _check(_load().sr_ref_producer_regress(
+        lr.ctypes.data, feat.ctypes.data, wconv.ctypes.data, None if bias is None else bias.ctypes.data, dict_.ctypes.data,
+        None if idx is None else idx.ctypes.data, None if gamma is None else gamma.ctypes.data, s, out.ctypes.data,
+        n, c, h, w, scale, k, D, cin, kc, flags, threads), "producer_regress")
+    return out

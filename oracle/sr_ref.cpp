@@ -29,6 +29,9 @@
  * responses built from the pinned dense regression, the LASSO against a library
  * solver and its optimality conditions, the re-fit against a library least-squares
  * solve, and the search against its stopping rules on hand-built problems.
+ * The producer of Phi (last convolution + pixel-shuffle, the survey's producer-fusion row) is pinned in
+ * tests/test_oracle_pins_producer.py against a library convolution and sub-pixel shuffle and against the pinned
+ * dense regression fed with its output.
  * No function here is parity-unpinned.
  */
 #include <algorithm>
@@ -770,6 +773,94 @@ int sr_ref_selection_search(const double* G_in, const double* b_in, double hh, i
         if (active[l]) { idx_out[cnt] = (uint8_t)l; gamma_out[cnt] = gtot[l]; ++cnt; }
     *count_out = cnt;
     if (steps_out) *steps_out = step;
+    return REF_OK;
+}
+
+/*
+ * The producer of Phi (Section II-A, stage 2: LaparNet is a stack of fusion blocks, pixel-shuffle layers and
+ * convolutions; only its last two layers are restated here, with seeded weights, as the survey's producer-fusion row).
+ * The LR feature map feat[n][h][w][cin] (binary16, channels last) goes through one convolution with kc x kc taps,
+ * zero padding kc/2, weights wconv[L r^2][cin][kc][kc] and bias[L r^2] (fp32), and a pixel-shuffle by r:
+ *     Phi_l(Y, X) = conv[l r^2 + (Y mod r) r + (X mod r)](Y div r, X div r)
+ * (the channel order of the common sub-pixel layer).  No activation follows: Phi are the raw outputs.
+ */
+static double producer_coef_at(const uint16_t* feat, const float* wconv, const float* bias, int cin, int kc, const Dims& d,
+                               int frame, int l, int Y, int X)
+{
+    const int r = d.r, pc = kc / 2;
+    const int o = l * r * r + (Y % r) * r + (X % r);
+    const int y0 = Y / r, x0 = X / r;
+    double acc = bias ? (double)bias[o] : 0.0;
+    for (int ci = 0; ci < cin; ++ci)
+        for (int dy = 0; dy < kc; ++dy)
+            for (int dx = 0; dx < kc; ++dx) {
+                const int yy = y0 + dy - pc, xx = x0 + dx - pc;
+                if (yy < 0 || yy >= d.h || xx < 0 || xx >= d.w) continue;            /* zero padding */
+                const double v = half_to_double(feat[(((int64_t)frame * d.h + yy) * d.w + xx) * cin + ci]);
+                acc += v * (double)wconv[(((int64_t)o * cin + ci) * kc + dy) * kc + dx];
+            }
+    return acc;
+}
+
+/* Phi[n][L][H][W] (fp64) from the feature map: the tensor the regression calls would otherwise read from memory. */
+int sr_ref_producer_coef(const void* feat, const float* wconv, const float* bias, double* phi, int n, int h, int w, int r,
+                         int L, int cin, int kc, int threads)
+{
+    Dims d{n, 1, h, w, r, 1, L};
+    if (!feat || !wconv || !phi) return REF_ERR_NULL;
+    if (int e = check_dims(d)) return e;
+    if (cin < 1 || kc < 1 || (kc % 2) == 0) return REF_ERR_UNSUPPORTED;
+    set_threads(threads);
+    const int H = d.H(), W = d.W();
+    for (int f = 0; f < n; ++f)
+        for (int l = 0; l < L; ++l) {
+#pragma omp parallel for schedule(static)
+            for (int Y = 0; Y < H; ++Y)
+                for (int X = 0; X < W; ++X)
+                    phi[(((int64_t)f * L + l) * H + Y) * W + X] =
+                        producer_coef_at((const uint16_t*)feat, wconv, bias, cin, kc, d, f, l, Y, X);
+        }
+    return REF_OK;
+}
+
+/*
+ * Stages 1-4 with Phi taken from the producer instead of memory: out[n][c][H][W] fp64.  With idx == NULL every atom is
+ * used (Eq. 2); with idx[s] (and gamma[s], or NULL for ones) the global subset of Section III-A, Eq. 6 / Eq. 9.
+ * Phi is not rounded to any storage type on the way: the fused path never stores it.
+ */
+int sr_ref_producer_regress(const float* lr, const void* feat, const float* wconv, const float* bias, const float* dict,
+                            const uint8_t* idx, const float* gamma, int s, double* out, int n, int c, int h, int w, int r,
+                            int k, int L, int cin, int kc, unsigned flags, int threads)
+{
+    Dims d{n, c, h, w, r, k, L};
+    if (!lr || !feat || !wconv || !dict || !out) return REF_ERR_NULL;
+    if (int e = check_dims(d)) return e;
+    if (cin < 1 || kc < 1 || (kc % 2) == 0) return REF_ERR_UNSUPPORTED;
+    if ((flags & REF_LUMA_ONLY) && c != 3) return REF_ERR_UNSUPPORTED;
+    if (idx && (s < 1 || s > L)) return REF_ERR_SHAPE;
+    set_threads(threads);
+    const int H = d.H(), W = d.W();
+    std::vector<double> U;
+    upsample_all(lr, d, U, flags);
+    const int natoms = idx ? s : L;
+    std::vector<int> atoms((size_t)natoms);
+    for (int q = 0; q < natoms; ++q) atoms[(size_t)q] = idx ? (int)idx[q] : q;
+    for (int q = 0; q < natoms; ++q)
+        if (atoms[(size_t)q] >= L) return REF_ERR_SHAPE;
+    for (int f = 0; f < n; ++f) {
+#pragma omp parallel for schedule(static)
+        for (int Y = 0; Y < H; ++Y) {
+            std::vector<double> wts((size_t)natoms), y((size_t)c);
+            for (int X = 0; X < W; ++X) {
+                for (int q = 0; q < natoms; ++q)
+                    wts[(size_t)q] = ((idx && gamma) ? (double)gamma[q] : 1.0) *
+                                     producer_coef_at((const uint16_t*)feat, wconv, bias, cin, kc, d, f, atoms[(size_t)q], Y, X);
+                auto patch = [&](int ch, int yy, int xx) { return U[(((int64_t)f * c + ch) * H + yy) * W + xx]; };
+                regress_pixel(d, dict, natoms, atoms.data(), wts.data(), Y, X, flags, patch, y.data());
+                for (int ch = 0; ch < c; ++ch) out[(((int64_t)f * c + ch) * H + Y) * W + X] = y[(size_t)ch];
+            }
+        }
+    }
     return REF_OK;
 }
 

@@ -140,3 +140,20 @@ def make_inputs(wl: Workload, seed: int = BASE_SEED):
 
 def num_threads() -> int:
     return int(_load().srg_num_threads())
+
+
+def make_producer(wl: Workload, cin: int = 32, kc: int = 3, seed: int = BASE_SEED):
+    """Inputs of the fused last layer: LR feature map feat [n][h][w][cin] float16 ~ N(0.5, 0.25), the weights of the
+    last convolution wconv [D r^2][cin][kc][kc] fp32 ~ N(0, sigma_w) and its bias [D r^2] fp32 ~ 1/D + N(0, 0.005),
+    with sigma_w chosen so that the coefficients the layer produces are distributed like the ones make_coef draws
+    (mean 1/D, standard deviation 0.05). Stand-ins for a trained network's features and weights."""
+    lib = _load()
+    r2 = wl.scale * wl.scale
+    feat = np.empty((wl.n, wl.h, wl.w, cin), dtype=np.float16)
+    lib.srg_fill_coef(seed, 1000, feat.ctypes.data, feat.size, 0.5, 0.25, 1)
+    wconv = np.empty((wl.D * r2, cin, kc, kc), dtype=np.float32)
+    sigma_w = 0.05 / float(np.sqrt(cin * kc * kc * (0.25 + 0.0625)))
+    lib.srg_fill_coef(seed, 1001, wconv.ctypes.data, wconv.size, 0.0, sigma_w, 0)
+    bias = np.empty((wl.D * r2,), dtype=np.float32)
+    lib.srg_fill_coef(seed, 1002, bias.ctypes.data, bias.size, 1.0 / wl.D, 0.005, 0)
+    return feat, wconv, bias
