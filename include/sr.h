@@ -263,6 +263,37 @@ int sr_tune_selected(const float* lr, const void* coef_or_sel, int coef_dtype, c
 void sr_tune_reset(void);
 
 /*
+ * Regression fused with the producer of the coefficients (Section II-A: the coefficient network ends in convolution
+ * and pixel-shuffle layers; Eq. 2-3 then use its output).  When that last layer is a plain convolution over an LR
+ * feature map followed by a pixel-shuffle by `scale`,
+ *     Phi_l(Y, X) = bias[o] + sum_{ci, dy, dx} feat[Y div r + dy - kc/2][X div r + dx - kc/2][ci] * wconv[o][ci][dy][dx],
+ *     o = l r^2 + (Y mod r) r + (X mod r)      (positions outside the map read zero),
+ * the coefficient tensor need never exist: F_i = Phi_i D is itself one convolution of the feature map with the weights
+ * folded with the dictionary.  sr_producer_fold builds those folded weights once per (network, dictionary);
+ * sr_producer_regress computes what sr_dict_regress_dense would compute on that Phi (or, after a fold with a subset,
+ * what sr_dict_regress_selected with SR_IDX_GLOBAL would), reading feat instead of coefficients.
+ *
+ *   wconv  [D*scale^2][cin][kc][kc] fp32 (device), bias [D*scale^2] fp32 (device) or NULL
+ *   dict   [D][k*k] fp32;  idx[s] / gamma[s] (device): an atom subset and its weights, or NULL / NULL for every atom
+ *          (gamma alone NULL: ones)
+ *   feat   [n][h][w][cin] binary16, channels last, 16-byte aligned
+ *   folded device buffer of sr_producer_folded_bytes(d, cin, kc) bytes, 16-byte aligned, owned by the caller; its
+ *          layout is private to the library and depends on d->scale, d->k, cin, kc (not on n, c, h, w, D)
+ *   out    [n][c][H][W], 16-byte aligned; fp32, or binary16 / uint8 with SR_OUT_F16 / SR_OUT_U8
+ * flags of sr_producer_regress: SR_CLAMP01, SR_UPSAMPLE_BILINEAR, SR_OUT_F16, SR_OUT_U8.
+ * Supported: scale 2 or 4, k in {3, 5, 7}, c <= 3, cin = 32, kc in {1, 3}; anything else is SR_ERR_UNSUPPORTED (there
+ * is no slower path behind this call) and sr_producer_folded_bytes returns 0.  The folded weights are rounded to
+ * binary16 (the bias keeps about 22 bits), feature values must be finite; results agree with the fp64 definition
+ * within the binary16 tolerance of the other calls.  Asynchronous on `stream`; device-side waits are bounded as in
+ * the other tensor-core calls (sr_device_status).
+ */
+size_t sr_producer_folded_bytes(const sr_dims* d, int cin, int kc);
+int sr_producer_fold(const float* wconv, const float* bias, const float* dict, const uint8_t* idx, const float* gamma,
+                     int s, void* folded, size_t folded_bytes, const sr_dims* d, int cin, int kc, void* stream);
+int sr_producer_regress(const float* lr, const void* feat, const void* folded, size_t folded_bytes, float* out,
+                        const sr_dims* d, int cin, int kc, uint32_t flags, void* stream);
+
+/*
  * Sustained issue rate of an arithmetic pipe of the current device, for the roofline of the kernels that are bound by
  * one (the selection networks by integer max/min, the general and subset regressions by fp32 multiply-add):
  * kind 0 = integer max/min, kind 1 = fp32 multiply-add.  Runs a register-only kernel a few times on `stream`,

@@ -22,7 +22,8 @@ SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA,
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
            "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival",
            "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes",
-           "sr_selection_gram_static", "sr_probe_rate", "sr_tune_dense", "sr_tune_selected", "sr_tune_reset")
+           "sr_selection_gram_static", "sr_probe_rate", "sr_tune_dense", "sr_tune_selected", "sr_tune_reset",
+           "sr_producer_folded_bytes", "sr_producer_fold", "sr_producer_regress")
 
 
 class sr_dims(ctypes.Structure):
@@ -84,6 +85,10 @@ def load_library() -> ctypes.CDLL:
         lib.sr_selection_search_scratch_bytes.argtypes = [ctypes.c_int32]
         lib.sr_selection_search_scratch_bytes.restype = sz
         lib.sr_selection_search.argtypes = [vp, vp, vp, f64, ctypes.c_int32, ctypes.POINTER(sr_search_opts), vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.sr_producer_folded_bytes.argtypes = [dp, i32, i32]
+        lib.sr_producer_folded_bytes.restype = sz
+        lib.sr_producer_fold.argtypes = [vp, vp, vp, vp, vp, i32, vp, sz, dp, i32, i32, vp]
+        lib.sr_producer_regress.argtypes = [vp, vp, vp, sz, vp, dp, i32, i32, u32, vp]
         lib.sr_status_string.argtypes = [i32]
         lib.sr_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -286,6 +291,45 @@ def sr_probe_rate(kind: int) -> float:
     v = ctypes.c_double(0.0)
     _check(load_library().sr_probe_rate(kind, _ptr(scratch), ctypes.byref(v), _stream()), "sr_probe_rate")
     return float(v.value)
+
+
+def sr_producer_fold(wconv, bias, dict_, scale: int, k: int, idx=None, gamma=None) -> torch.Tensor:
+    """Folds the dictionary (every atom, or the subset idx with weights gamma) into the last convolution's weights
+    wconv [D*scale^2][cin][kc][kc] and bias; returns the folded block sr_producer_regress takes."""
+    wconv, dict_ = _dev(wconv, torch.float32, "wconv"), _dev(dict_, torch.float32, "dict")
+    bias = None if bias is None else _dev(bias, torch.float32, "bias")
+    idx = None if idx is None else _dev(idx, torch.uint8, "idx")
+    gamma = None if gamma is None else _dev(gamma, torch.float32, "gamma")
+    cout, cin, kc, kc2 = wconv.shape
+    D = dict_.shape[0]
+    if kc2 != kc or cout != D * scale * scale or dict_.shape[1] != k * k or (bias is not None and bias.numel() != cout):
+        raise ValueError("shapes of wconv / bias / dict do not agree")
+    d = sr_dims(1, 1, 1, 1, scale, k, D)
+    lib = load_library()
+    nbytes = int(lib.sr_producer_folded_bytes(ctypes.byref(d), cin, kc))
+    if nbytes == 0:
+        raise SrError(SR_ERR_UNSUPPORTED, "sr_producer_folded_bytes")
+    folded = torch.empty(nbytes, dtype=torch.uint8, device=wconv.device)
+    _check(lib.sr_producer_fold(_ptr(wconv), _ptr(bias), _ptr(dict_), _ptr(idx), _ptr(gamma), 0 if idx is None else idx.numel(),
+                                _ptr(folded), nbytes, ctypes.byref(d), cin, kc, _stream()), "sr_producer_fold")
+    return folded
+
+
+def sr_producer_regress(lr, feat, folded, scale: int, k: int, D: int, kc: int, flags: int = 0, out=None) -> torch.Tensor:
+    """Dense (or folded-subset) regression with the coefficients computed on the fly from the LR feature map
+    feat [n][h][w][cin] (float16, channels last) and the folded weights."""
+    lr, feat = _dev(lr, torch.float32, "lr"), _dev(feat, torch.float16, "feat")
+    folded = _dev(folded, torch.uint8, "folded")
+    n, c, h, w = lr.shape
+    if tuple(feat.shape[:3]) != (n, h, w):
+        raise ValueError("feat must be [n][h][w][cin]")
+    cin = feat.shape[3]
+    if out is None:
+        out = torch.empty((n, c, h * scale, w * scale), dtype=_out_dtype(flags), device=lr.device)
+    d = sr_dims(n, c, h, w, scale, k, D)
+    _check(load_library().sr_producer_regress(_ptr(lr), _ptr(feat), _ptr(folded), folded.numel(), _ptr(out), ctypes.byref(d), cin, kc,
+                                              flags, _stream()), "sr_producer_regress")
+    return out
 
 
 def _tune_dict(res: sr_tune_result) -> dict:

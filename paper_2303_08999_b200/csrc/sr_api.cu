@@ -9,6 +9,7 @@
 
 #include "sr_common.cuh"
 #include "sr_regress_subset.cuh"
+#include "sr_producer.cuh"
 #include "sr_regress_tc.cuh"
 #include "sr_selection.cuh"
 #include "sr_umma.cuh"
@@ -474,6 +475,42 @@ const char* sr_status_string(int status)
 }
 
 int64_t sr_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+size_t sr_producer_folded_bytes(const sr_dims* d, int cin, int kc)
+{
+    if (!d || check_dims(d, true) != SR_OK) return 0;
+    return producer_folded_bytes(make_problem(d, d->D, 0u), ProducerShape{cin, kc});
+}
+
+int sr_producer_fold(const float* wconv, const float* bias, const float* dict, const uint8_t* idx, const float* gamma,
+                     int s, void* folded, size_t folded_bytes, const sr_dims* d, int cin, int kc, void* stream)
+{
+    if (!wconv || !dict || !folded || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (gamma && !idx) return SR_ERR_UNSUPPORTED;
+    if (idx && (s < 1 || s > d->D)) return SR_ERR_SHAPE;
+    const Problem pb = make_problem(d, d->D, 0u);
+    const ProducerShape ps{cin, kc};
+    if (!producer_supported(pb, ps)) return SR_ERR_UNSUPPORTED;
+    if (folded_bytes < producer_folded_bytes(pb, ps)) return SR_ERR_SHAPE;
+    if (!aligned(wconv, 4) || !aligned(dict, 4) || (bias && !aligned(bias, 4)) || (gamma && !aligned(gamma, 4)) || !aligned(folded, 16))
+        return SR_ERR_ALIGN;
+    return launch_producer_fold(wconv, bias, dict, idx, gamma, s, folded, pb, ps, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
+
+int sr_producer_regress(const float* lr, const void* feat, const void* folded, size_t folded_bytes, float* out,
+                        const sr_dims* d, int cin, int kc, uint32_t flags, void* stream)
+{
+    if (!lr || !feat || !folded || !out || !d) return SR_ERR_NULL;
+    if (int e = check_dims(d, true)) return e;
+    if (flags & ~(uint32_t)(SR_CLAMP01 | SR_UPSAMPLE_BILINEAR | SR_OUT_F16 | SR_OUT_U8) || bad_out_flags(flags, d)) return SR_ERR_UNSUPPORTED;
+    const Problem pb = make_problem(d, d->D, flags);
+    const ProducerShape ps{cin, kc};
+    if (!producer_supported(pb, ps)) return SR_ERR_UNSUPPORTED;
+    if (folded_bytes < producer_folded_bytes(pb, ps)) return SR_ERR_SHAPE;
+    if (!aligned(lr, 4) || !aligned(feat, 16) || !aligned(folded, 16) || !aligned(out, 16)) return SR_ERR_ALIGN;
+    return launch_producer_regress(lr, feat, folded, out, pb, ps, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
+}
 
 int sr_probe_rate(int kind, void* scratch8, double* lane_ops_per_s, void* stream)
 {
