@@ -850,11 +850,26 @@ int sr_ref_producer_regress(const float* lr, const void* feat, const float* wcon
     for (int f = 0; f < n; ++f) {
 #pragma omp parallel for schedule(static)
         for (int Y = 0; Y < H; ++Y) {
-            std::vector<double> wts((size_t)natoms), y((size_t)c);
+            std::vector<double> wts((size_t)natoms), y((size_t)c), xwin((size_t)cin * kc * kc);
             for (int X = 0; X < W; ++X) {
-                for (int q = 0; q < natoms; ++q)
-                    wts[(size_t)q] = ((idx && gamma) ? (double)gamma[q] : 1.0) *
-                                     producer_coef_at((const uint16_t*)feat, wconv, bias, cin, kc, d, f, atoms[(size_t)q], Y, X);
+                /* the feature values under the kernel at this pixel's LR position, widened once ([ci][dy][dx], zeros
+                 * outside the map); then Phi_l as in producer_coef_at, one dot product per atom */
+                const int pc = kc / 2, y0 = Y / r, x0 = X / r;
+                for (int ci = 0; ci < cin; ++ci)
+                    for (int dy = 0; dy < kc; ++dy)
+                        for (int dx = 0; dx < kc; ++dx) {
+                            const int yy = y0 + dy - pc, xx = x0 + dx - pc;
+                            const bool inside = yy >= 0 && yy < h && xx >= 0 && xx < w;
+                            xwin[((size_t)ci * kc + dy) * kc + dx] =
+                                inside ? half_to_double(((const uint16_t*)feat)[(((int64_t)f * h + yy) * w + xx) * cin + ci]) : 0.0;
+                        }
+                for (int q = 0; q < natoms; ++q) {
+                    const int o = atoms[(size_t)q] * r * r + (Y % r) * r + (X % r);
+                    const float* wrow = wconv + (int64_t)o * cin * kc * kc;
+                    double phi = bias ? (double)bias[o] : 0.0;
+                    for (int i = 0; i < cin * kc * kc; ++i) phi += xwin[(size_t)i] * (double)wrow[i];
+                    wts[(size_t)q] = ((idx && gamma) ? (double)gamma[q] : 1.0) * phi;
+                }
                 auto patch = [&](int ch, int yy, int xx) { return U[(((int64_t)f * c + ch) * H + yy) * W + xx]; };
                 regress_pixel(d, dict, natoms, atoms.data(), wts.data(), Y, X, flags, patch, y.data());
                 for (int ch = 0; ch < c; ++ch) out[(((int64_t)f * c + ch) * H + Y) * W + X] = y[(size_t)ch];

@@ -52,6 +52,7 @@ template <int R, int K> struct PG {
     static constexpr int TH = R * TLH;                 // HR rows of a tile
     static constexpr int RG = (R == 4 && 2 * R * kk <= 256) ? 2 : 1;   // phase rows per pass
     static constexpr int G = R / RG;                   // passes per tile
+    static constexpr bool SPLIT = RG == 2;             // both epilogue groups work on every pass, one phase row each
     static constexpr int FW = R * K;                   // taps of one patch row for the r pixels of an HR row of the block
     static constexpr int FWP = (FW + 3) & ~3;          // padded so that tensor-memory loads stay naturally aligned
     static constexpr int NCOL = RG * K * FWP;          // accumulator columns of a pass
@@ -168,9 +169,10 @@ template <> __device__ __forceinline__ void store_pixels<2, uint8_t>(uint8_t* ds
 // One pass of one tile for one thread: the RG phase rows of pass g for the r x r block of this thread's LR pixel.
 //   u_px:   the up-sampled tile at (channel 0, row 0, this block's first column); planes u_plane floats apart
 //   out_px: channel 0, first row of the tile, this block's first pixel; channels HW elements apart
+//   only_ryl: the one phase row of the pass this thread takes (split passes), or -1 for all of them
 template <int R, int K, typename OutT>
 __device__ __forceinline__ void epilogue_pass(const float* u_px, int u_plane, OutT* out_px, int64_t HW, int W, int C, int g,
-                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01)
+                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01, int only_ryl)
 {
     using G = PG<R, K>;
     constexpr int UWIN = R + K - 1;                 // neighbouring values of a patch row the r pixels share
@@ -178,6 +180,7 @@ __device__ __forceinline__ void epilogue_pass(const float* u_px, int u_plane, Ou
     constexpr int NV = (UWIN + UV - 1) / UV;
 #pragma unroll
     for (int ryl = 0; ryl < G::RG; ++ryl) {
+        if (only_ryl >= 0 && ryl != only_ryl) continue;
         const int yt = R * yl + g * G::RG + ryl;    // row inside the tile
         float acc[kMaxC][R];
 #pragma unroll
@@ -251,7 +254,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
     if (tid == 0) {
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.b_full[i], 1); mbar_init(&ctl.b_empty[i], 1); }
         for (int i = 0; i < kMaxSteps; ++i) { mbar_init(&ctl.a_full[i], 1); mbar_init(&ctl.a_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], G::SPLIT ? 8 : 4); }
         mbar_init(&ctl.lr_full, 32);
         mbar_init(&ctl.lr_empty, 1);
         mbar_init(&ctl.drain, 1);
@@ -401,7 +404,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
         const int yl = m / G::TLW, xl = m - yl * G::TLW;
         const int64_t HW = (int64_t)pb.H * pb.W;
         const bool clamp01 = (pb.flags & SR_CLAMP01) != 0;
-        const uint32_t tmem_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)e * 256u;
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int et = tid - kUtilThreads;
         const int tc4 = p.g.tcols >> 2;
         const int v_lane = fast_div(et, tc4, p.g.tc4_magic), v_i4 = (et - v_lane * tc4) * 4, v_lanes = kEpiThreads / tc4;
@@ -423,14 +426,18 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             named_barrier_sync(1, kEpiThreads);              // the U tile is complete
             const bool in_x = w.x0 + R * xl < pb.W;
             OutT* out_px = reinterpret_cast<OutT*>(p.out) + (int64_t)w.f * C * HW + (int64_t)w.y0 * pb.W + w.x0 + R * xl;
-            for (int g = e; g < G::G; g += 2, ++pe) {
-                ok = mbar_wait_leader(&ctl.acc_full[e], pe & 1, wc, false);
+            // split passes: both groups take every pass (buffers alternate), group e the phase row e of it;
+            // otherwise group e takes the passes with g % 2 == e, which always land in buffer e
+            for (int g = G::SPLIT ? 0 : e; g < G::G; g += G::SPLIT ? 1 : 2, ++pe) {
+                const uint32_t buf = G::SPLIT ? (pe & 1u) : (uint32_t)e;
+                ok = mbar_wait_leader(&ctl.acc_full[buf], (G::SPLIT ? (pe >> 1) : pe) & 1u, wc, false);
                 if (!ok) break;
                 tc_fence_after_sync();
-                epilogue_pass<R, K, OutT>(sU + R * xl, u_plane, out_px, HW, pb.W, C, g, tmem_lane, yl, w.rows, in_x, clamp01);
+                epilogue_pass<R, K, OutT>(sU + R * xl, u_plane, out_px, HW, pb.W, C, g, tmem_lane + buf * 256u, yl, w.rows, in_x,
+                                          clamp01, G::SPLIT ? e : -1);
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl.acc_empty[e]);   // this warp has read its lanes of the buffer
+                if (lane == 0) mbar_arrive(&ctl.acc_empty[buf]);   // this warp has read its lanes of the buffer
             }
             // a failed wait is agreed on at the next tile's barrier, so that nobody is left waiting there
         }

@@ -121,3 +121,20 @@ def test_a_lost_copy_times_out_and_the_next_call_is_correct():
         sr.sr_test_lose_arrival(0)
     again = sr.sr_producer_regress(dlr, dfe, folded, wl.scale, wl.k, wl.D, 3)
     assert torch.equal(again, good)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3"])
+def test_full_size_whole_frame(name):
+    """The 1080p x4 frame of the benchmark and one frame of the 4K x2 batch, element by element over the whole output,
+    in the launch configuration bench.py times (signed, asymmetric dictionary)."""
+    from dataclasses import replace
+    wl = replace(sr_inputs.CONFIGS[name], n=1)
+    lr, dict_, _ = sr_inputs.make_inputs(replace(wl, D=1))      # the coefficient tensor is not needed here
+    dict_ = signed_asymmetric_dictionary(sr_inputs.make_dictionary(wl.D, wl.k))
+    feat, wconv, bias = sr_inputs.make_producer(wl, cin=32, kc=3)
+    folded = sr.sr_producer_fold(dev(wconv), dev(bias), dev(dict_), wl.scale, wl.k)
+    got = sr.sr_producer_regress(dev(lr), torch.from_numpy(feat).cuda(), folded, wl.scale, wl.k, wl.D, 3, sr.SR_CLAMP01)
+    want = oracle.producer_regress(lr, feat, wconv, bias, dict_, wl.scale, wl.k, flags=oracle.CLAMP01)
+    err = np.abs(host(got) - want).max()
+    assert err <= TIGHT, err
+    assert sr.sr_device_status() == 0
