@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the dictionary-regression hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg0|cfg1|cfg2|cfg3|cfg4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg0|cfg1|cfg2|cfg3|cfg4|producer]
 
 One step = one pass of the whole hot path over one frame batch of the workload (default: the
 1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. six library
@@ -28,6 +28,9 @@ with the per-path times and roofline fractions, the clocks seen during its timed
 small sample (`--points r3_D72_k5` restricts the sweep). Every path's roofline is the slowest of its bytes at the
 measured HBM bandwidth, its selection-network operations at the measured integer max/min rate and its multiply-adds
 at the measured fp32 rate (both rates are measured at start-up by the library's probe kernels).
+`--workload producer` times the regression fused with the last layer of the coefficient network (sr_producer_regress, one
+call per step on the cfg1 frame, features [n][h][w][32] binary16, 3x3 convolution): its roofline is the folded
+convolution's tensor-core work against the measured dense bf16 rate.
 """
 from __future__ import annotations
 
@@ -256,10 +259,41 @@ def time_oracle(wl, lr, dict_, coef, S, gamma, budget_s: float = 20.0):
                       f"step, {dt:.2f} s of fp64 CPU work"}
 
 
-def run_reference(args, wl):
+def run_reference_producer(args, wl):
+    """Reference arm of `--workload producer`: the oracle's producer + regression on a band of LR rows per step."""
+    import oracle
+    import sr_inputs
+    one = sr_inputs.Workload(wl.name, 1, wl.c, wl.h, wl.w, wl.scale, wl.D, wl.k, wl.coef_dtype, wl.s)
+    lr, dict_ = sr_inputs.make_lr(one), sr_inputs.make_dictionary(wl.D, wl.k)
+    feat, wconv, bias = sr_inputs.make_producer(one, PRODUCER_CIN, PRODUCER_KC)
+    call = lambda rows: oracle.producer_regress(lr[:, :, :rows].copy(), feat[:, :rows].copy(), wconv, bias, dict_, wl.scale, wl.k,
+                                                flags=oracle.CLAMP01)
+    t0 = time.perf_counter()
+    call(4)
+    rate = 4 / (time.perf_counter() - t0)
+    rows = int(max(1, min(wl.h, 120.0 / max(1, args.steps + args.warmup) * rate)))
+    for _ in range(args.warmup):
+        call(rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        call(rows)
+    dt = time.perf_counter() - t0
+    value = args.steps * rows * wl.scale * wl.W / dt / 1e6
+    sample = f"top {rows} of {wl.h} LR rows of one frame per step, producer + regression"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "MP/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": "producer (cfg1 frame, 32 feature channels, 3x3 convolution)"},
+        "cpu_baseline": {"value": value, "unit": "MP/s", "cores": oracle.max_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "MP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def run_reference(args, wl, producer: bool = False):
     """The reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    if producer:
+        return run_reference_producer(args, wl)
     import oracle
     import numpy as np
     import sr_inputs
@@ -496,6 +530,156 @@ def run_workload(wl, args, active, peaks, dist, rank, world, local_rank, steps: 
     }
 
 
+PRODUCER_CIN, PRODUCER_KC = 32, 3
+
+
+def producer_flops(wl, cin: int, kc: int) -> float:
+    """Tensor-core work of the fused last layer per launch: the folded convolution, 2 x LR pixels x (kc^2 cin) x
+    (r^2 k^2) (the bias K-step and the padding columns are not counted)."""
+    return 2.0 * wl.n * wl.h * wl.w * (kc * kc * cin) * (wl.scale ** 2 * wl.k ** 2)
+
+
+def producer_bytes(wl, cin: int) -> float:
+    """Bytes that must cross HBM per launch: feature map and LR frame read once, output written once."""
+    return float(wl.n * wl.h * wl.w * (cin * 2 + 4 * wl.c) + wl.npix * 4 * wl.c)
+
+
+def time_oracle_producer(wl, lr, feat, wconv, bias, dict_, budget_s: float):
+    import oracle
+    rows = 4
+    t0 = time.perf_counter()
+    oracle.producer_regress(lr[:1, :, :rows], feat[:1, :rows], wconv, bias, dict_, wl.scale, wl.k, flags=oracle.CLAMP01)
+    rate = rows / (time.perf_counter() - t0)
+    rows = int(max(4, min(wl.h, budget_s * rate)))
+    t0 = time.perf_counter()
+    oracle.producer_regress(lr[:1, :, :rows].copy(), feat[:1, :rows].copy(), wconv, bias, dict_, wl.scale, wl.k, flags=oracle.CLAMP01)
+    dt = time.perf_counter() - t0
+    px = rows * wl.scale * wl.W
+    return {"value": px / dt / 1e6, "unit": "MP/s", "cores": oracle.max_threads(), "kind": "oracle",
+            "sample": f"top {rows} of {wl.h} LR rows of one frame ({px} HR pixels), producer + regression, {dt:.2f} s of fp64 CPU work"}
+
+
+def run_producer(wl, args, dist, rank, world, local_rank, steps: int, warmup: int):
+    """`--workload producer`: the regression fused with the last convolution + pixel-shuffle of the coefficient network
+    (sr_producer_regress) on the 1080p x4 frame; one step = one call. The dictionary is folded into the layer's
+    weights once, outside the timed region (it depends on the network and the dictionary, not on the frame)."""
+    import numpy as np
+    import torch
+    import paper_2303_08999_b200 as sr
+    import sr_inputs
+
+    cin, kc = PRODUCER_CIN, PRODUCER_KC
+    seed = rank_seed(sr_inputs.BASE_SEED, rank)
+    lr = sr_inputs.make_lr(wl, seed)
+    dict_ = sr_inputs.make_dictionary(wl.D, wl.k, seed)
+    feat, wconv, bias = sr_inputs.make_producer(wl, cin, kc, seed)
+    h_lr, h_feat = torch.from_numpy(lr).pin_memory(), torch.from_numpy(feat).pin_memory()
+    folded = sr.sr_producer_fold(*(torch.from_numpy(a).cuda() for a in (wconv, bias, dict_)), wl.scale, wl.k)
+    shape_out = (wl.n, wl.c, wl.H, wl.W)
+    per_set = feat.nbytes + lr.nbytes + 4 * wl.n * wl.c * wl.H * wl.W
+    nsets = int(max(3, min(96, -(-2 * 126 * 1024 * 1024 // per_set))))
+    sets = [{"lr": h_lr.cuda(), "feat": h_feat.cuda(), "out": torch.empty(shape_out, dtype=torch.float32, device="cuda")}
+            for _ in range(nsets)]
+    flags = sr.SR_CLAMP01
+
+    def step(b, out=None):
+        sr.sr_producer_regress(b["lr"], b["feat"], folded, wl.scale, wl.k, wl.D, kc, flags, out=b["out"] if out is None else out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    if sampler:
+        sampler.wait_first_sample()
+    for i in range(warmup):
+        step(sets[i % nsets])
+    barrier()
+    # the kernel's own duration: an event on both sides of every launch (not the headline)
+    evs = []
+    for i in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); step(sets[i % nsets]); b.record()
+        evs.append((a, b))
+    barrier()
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+    launches0 = sr.sr_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    wall0 = time.time()
+    t0.record()
+    for i in range(steps):
+        step(sets[i % nsets])
+    t1.record()
+    barrier()
+    wall1 = time.time()
+    elapsed_ms = max_over_ranks(t0.elapsed_time(t1), dist, "cuda")
+    launches = sr.sr_launch_count() - launches0
+    clocks = sampler.stop(wall0, wall1) if sampler else None
+    if sr.sr_device_status() != 0:
+        raise SystemExit("device status word reports an expired wait")
+
+    # end to end: pinned host -> device copies of the LR frame and the feature map, device -> host copy of the result
+    e2e = None
+    if not args.no_e2e:
+        from paper_2303_08999_b200.hostpipe import HostPipeline
+        h_out = {"out": torch.empty(shape_out, dtype=torch.float32).pin_memory()}
+        pipe = HostPipeline({"lr": (tuple(h_lr.shape), h_lr.dtype), "feat": (tuple(h_feat.shape), h_feat.dtype)},
+                            {"out": (shape_out, torch.float32)}, depth=2)
+        e2e_steps = max(3, min(steps, 20))
+        fn = lambda: pipe.submit({"lr": h_lr, "feat": h_feat}, h_out, lambda i, o: step(i, o["out"]))
+        fn(); pipe.drain(); barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e2e_steps):
+            fn()
+        pipe.drain()
+        b.record()
+        barrier()
+        ms = max_over_ranks(a.elapsed_time(b), dist, "cuda")
+        e2e = {"value": whole_job_value(world, wl.npix, e2e_steps, ms), "unit": "MP/s",
+               "h2d_bytes_per_step": lr.nbytes + feat.nbytes, "d2h_bytes_per_step": 4 * wl.n * wl.c * wl.H * wl.W,
+               "steps": e2e_steps, "how": "HostPipeline, depth 2: copy-in, kernel and copy-out on three streams"}
+    if rank != 0:
+        return None
+    tf_peak, tf_kind = load_tensor_peak()
+    fl = producer_flops(wl, cin, kc)
+    by = producer_bytes(wl, cin)
+    sec = kernel_ms * 1e-3
+    roofline = {"bound": "tensor", "kernel": "producer_regress_kernel", "achieved": fl / sec / 1e12, "peak": tf_peak, "unit": "TFLOP/s",
+                "frac": fl / sec / 1e12 / tf_peak, "peak_kind": f"of {tf_kind} (dense bf16 burst; binary16 runs at the same nominal rate)",
+                "traffic": None, "roofline_us": fl / (tf_peak * 1e12) * 1e6, "kernel_us": kernel_ms * 1e3,
+                "hbm_bytes": by, "hbm_frac": by / sec / 1e9 / load_peaks()[0],
+                "bytes_a_separate_coefficient_tensor_would_add": 2.0 * wl.D * 2 * wl.npix}
+    cpu = None if args.no_cpu_baseline else time_oracle_producer(wl, lr, feat, wconv, bias, dict_, 15.0)
+    return {
+        "metric": METRIC, "value": whole_job_value(world, wl.npix, steps, elapsed_ms), "unit": "MP/s", "n_gpus": world,
+        "steps": steps, "warmup": warmup, "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 operands, f32 accumulate", "data": "synthetic",
+        "config": {"workload": f"producer: LR {wl.n}x{wl.c}x{wl.h}x{wl.w} fp32 + features [n][h][w][{cin}] f16, last layer "
+                               f"{kc}x{kc} conv -> {wl.D}x{wl.scale}^2 channels + pixel-shuffle x{wl.scale}, D={wl.D} atoms of "
+                               f"{wl.k}x{wl.k}, folded; one sr_producer_regress call per step",
+                   "l2": f"{nsets} sets of (features, LR frame, output) rotate between steps; together larger than twice the 126 MB L2"},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
+    }
+
+
+def load_tensor_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        if "bf16_tflops" in d:
+            return float(d["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -509,7 +693,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     sweep = args.workload == "cfg4"
-    steps = args.steps if args.steps is not None else (20 if sweep else (30 if args.workload == "cfg3" else 300))
+    steps = args.steps if args.steps is not None else (20 if sweep else (30 if args.workload == "cfg3" else (3000 if args.workload == "producer" else 300)))
     warmup = args.warmup if args.warmup is not None else (3 if sweep or args.workload == "cfg3" else 10)
     if args.impl == "ours":
         warmup = max(warmup, 3)
@@ -520,14 +704,17 @@ def main():
 
     import sr_inputs
     from dataclasses import replace
-    if sweep:
+    producer = args.workload == "producer"
+    if producer:
+        wls = [sr_inputs.CONFIGS["cfg1"]]
+    elif sweep:
         want = [w for w in args.points.split(",") if w]
         wls = [replace(p, s=s) for p in sr_inputs.cfg4_points() for s in (4, 8, 16)
                if s <= p.D and (not want or any(w in p.name for w in want))]
     else:
         wls = [sr_inputs.CONFIGS[args.workload]]
     if args.impl == "reference":
-        run_reference(args, sr_inputs.CONFIGS[args.workload])    # the sweep's reference arm times its anchor point
+        run_reference(args, wls[0] if producer else sr_inputs.CONFIGS[args.workload], producer)   # the sweep's reference arm times its anchor point
         return
 
     import torch
@@ -547,6 +734,11 @@ def main():
     peaks = measure_peaks(sr)
     default_line = args.workload in ("cfg1", "cfg2")
     for wl in wls:
+        if producer:
+            line = run_producer(wl, args, dist, rank, world, local_rank, steps, warmup)
+            if line is not None:
+                print(json.dumps(line), flush=True)
+            continue
         line = run_workload(wl, args, active, peaks, dist, rank, world, local_rank, steps, warmup,
                             with_e2e=default_line and not args.no_e2e,
                             cpu_budget_s=0.0 if args.no_cpu_baseline else (1.0 if sweep else 20.0))
