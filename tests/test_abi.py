@@ -98,6 +98,18 @@ def test_validation_errors_come_back_before_any_launch(lib):
     assert selected(_dims(c=1), 4, flags=api.SR_LUMA_ONLY) == api.SR_ERR_UNSUPPORTED
     assert lib.sr_device_status(None, None) == api.SR_ERR_NULL
 
+    # the producer-fused calls: pointers and shapes are validated before anything touches the device; without a
+    # device that can run the kernel the size query answers 0 and the calls refuse the shape
+    d = _dims(scale=4)
+    assert lib.sr_producer_fold(None, None, FAKE, None, None, 0, FAKE, 16, ctypes.byref(d), 32, 3, None) == api.SR_ERR_NULL
+    assert lib.sr_producer_fold(FAKE, None, FAKE, None, FAKE, 0, FAKE, 16, ctypes.byref(d), 32, 3, None) == api.SR_ERR_UNSUPPORTED  # gamma without idx
+    assert lib.sr_producer_fold(FAKE, None, FAKE, FAKE, None, 99, FAKE, 16, ctypes.byref(d), 32, 3, None) == api.SR_ERR_SHAPE
+    assert lib.sr_producer_regress(FAKE, None, FAKE, 16, FAKE, ctypes.byref(d), 32, 3, 0, None) == api.SR_ERR_NULL
+    assert lib.sr_producer_regress(FAKE, FAKE, FAKE, 16, FAKE, ctypes.byref(d), 32, 3, api.SR_LUMA_ONLY, None) == api.SR_ERR_UNSUPPORTED
+    assert lib.sr_producer_regress(FAKE, FAKE, FAKE, 16, FAKE, ctypes.byref(_dims(scale=3)), 32, 3, 0, None) == api.SR_ERR_UNSUPPORTED
+    assert lib.sr_producer_folded_bytes(ctypes.byref(_dims(scale=3)), 32, 3) == 0
+    assert lib.sr_producer_folded_bytes(ctypes.byref(d), 16, 3) == 0
+
 
 def test_binding_refuses_cpu_tensors():
     import torch
