@@ -572,8 +572,12 @@ Plan make_plan_rk(const Problem& pb, const ProducerShape& ps)
     pl.ntaps = ps.kc * ps.kc;
     pl.passes = G::G;
     Geom g;
+    // the shared memory is planned for three channels whatever the frame has, so that the layout of the folded block
+    // (taps per step) depends on scale, k and the layer only, as the header promises
+    Problem pb3 = pb;
+    pb3.c = kMaxC;
     const size_t fixed = 1024 /* alignment slack */ + 32 + (size_t)pl.ntaps * kTapBytes + kOnesBytes +
-                         plan_geom(g, pb, G::TH, nullptr) * sizeof(float);
+                         plan_geom(g, pb3, G::TH, nullptr) * sizeof(float);
     const size_t per_cta = (size_t)di.smem_optin - kStaticReserve;
     // a step = the taps of one kernel row when two such stages fit, else a single tap
     for (int tps = ps.kc; tps >= 1; tps = (tps > 1 ? 1 : 0)) {
