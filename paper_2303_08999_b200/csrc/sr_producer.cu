@@ -24,8 +24,8 @@
 // vector loads) and accumulates r x c outputs; r consecutive output pixels leave as one vector store. Two groups of four
 // warps take alternate passes. The up-sampled tile is built per tile by the epilogue warps (stage 1, Section II-A;
 // shared code with the other regression kernels).
-// Warps: 0 producer (TMA + bulk copies, one thread), 1 MMA issuer (one thread; owns tensor memory), 2 LR-window
-// prefetch, 3 idle, 4-7 / 8-11 epilogue groups. One CTA per SM (512 TMEM columns), persistent over tiles.
+// Warps: 0 producer (TMA + bulk copies, one thread), 1 MMA issuer (one thread; owns tensor memory), 2-3 LR-window
+// prefetch (two windows ahead), 4-7 / 8-11 epilogue groups. One CTA per SM (512 TMEM columns), persistent over tiles.
 // Every wait is bounded; on expiry the CTA raises its abort flag, sets the device status word, drains and returns.
 #include "sr_ptx.cuh"
 #include "sr_producer.cuh"
@@ -43,25 +43,25 @@ constexpr int kTapBytes = 128 * kCin * 2;   // one tap of the A operand: 128 pix
 constexpr int kOnesBytes = 128 * 16 * 2;    // the constant A tile of the bias K-step
 constexpr int kUtilThreads = 128, kEpiThreads = 256, kThreads = kUtilThreads + kEpiThreads;
 constexpr int kMaxSteps = 9, kMaxStages = 4, kMaxC = 3;
-constexpr int kMmaWarp = 1, kLrWarp = 2;
+constexpr int kMmaWarp = 1, kLrWarp = 2, kLrThreads = 64;   // warps 2 and 3 prefetch LR windows
 
 template <int R, int K> struct PG {
     static constexpr int kk = K * K, P = (K - 1) / 2;
     static constexpr int TLW = TW / R;                 // LR columns of a tile
     static constexpr int TLH = 128 / TLW;              // LR rows of a tile
     static constexpr int TH = R * TLH;                 // HR rows of a tile
-    static constexpr int RG = (R == 4 && 2 * R * kk <= 256) ? 2 : 1;   // phase rows per pass
-    static constexpr int G = R / RG;                   // passes per tile
-    static constexpr bool SPLIT = RG == 2;             // both epilogue groups work on every pass, one phase row each
     static constexpr int FW = R * K;                   // taps of one patch row for the r pixels of an HR row of the block
     static constexpr int FWP = (FW + 3) & ~3;          // padded so that tensor-memory loads stay naturally aligned
+    static constexpr int RG = (R % 2 == 0 && 2 * K * FWP <= 256) ? 2 : 1;   // phase rows per pass (N <= 256)
+    static constexpr int G = R / RG;                   // passes per tile
+    static constexpr bool SPLIT = RG == 2;             // both epilogue groups work on every pass, one phase row each
     static constexpr int NCOL = RG * K * FWP;          // accumulator columns of a pass
     static constexpr int NG = (NCOL + 15) / 16 * 16;   // N of the MMA
     static constexpr int UW = tile_uw(P), UW4 = UW / 4;
     static constexpr int LBO_B = NG * 16;              // bytes between the two 8-channel groups of a K-step of B
     static constexpr int BIAS_BYTES = 2 * LBO_B;       // one K-step
     static constexpr int TAP_B_BYTES = 4 * LBO_B;      // two K-steps (32 channels)
-    static_assert(TLW * TLH == 128 && (G % 2) == 0 && NG <= 256, "tile or pass shape");
+    static_assert(TLW * TLH == 128 && (SPLIT || (G % 2) == 0) && NG <= 256, "tile or pass shape");
     // accumulator column of tap (a, b) for pixel rx of phase row ryl
     __host__ __device__ static constexpr int col_of(int ryl, int a, int rx, int b) { return (ryl * K + a) * FWP + rx * K + b; }
 };
@@ -75,6 +75,7 @@ struct ProdParams {
     int kc, ntaps;
     int tps, nsteps;          // taps per pipeline step, steps per pass
     int stages;
+    int resident;             // 1: every weight stage of a tile has its own slot; the weights are loaded once per CTA
     uint32_t stage_bytes;
     long long wait_cycles;
     int inject_lost_arrival;
@@ -84,7 +85,7 @@ struct __align__(16) Ctl {
     uint64_t b_full[kMaxStages], b_empty[kMaxStages];
     uint64_t a_full[kMaxSteps], a_empty[kMaxSteps];
     uint64_t acc_full[2], acc_empty[2];
-    uint64_t lr_full, lr_empty;
+    uint64_t lr_full[2], lr_empty[2];
     uint64_t drain;
     uint32_t tmem_base;
     WaitCtx wait;
@@ -247,16 +248,16 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
     uint8_t* sB = sOnes + kOnesBytes;                             // [stages][stage_bytes]
     float* sU = reinterpret_cast<float*>(sB + (size_t)p.stages * p.stage_bytes);   // [C][uh][UW]
     float* sV = sU + C * p.g.uh * G::UW;                          // [C][uh][tcols]
-    float* sL = sV + C * p.g.uh * p.g.tcols;                      // [C * trows][tcols]
-    const int dyn_bytes = (int)((uint8_t*)(sL + C * p.g.trows * p.g.tcols) - smem) + 32;
+    float* sL = sV + C * p.g.uh * p.g.tcols;                      // [2 buffers][C * trows][tcols]
+    const int l_tile = C * p.g.trows * p.g.tcols;                 // floats of one LR window
+    const int dyn_bytes = (int)((uint8_t*)(sL + 2 * l_tile) - smem) + 32;
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&ctl.b_full[i], 1); mbar_init(&ctl.b_empty[i], 1); }
         for (int i = 0; i < kMaxSteps; ++i) { mbar_init(&ctl.a_full[i], 1); mbar_init(&ctl.a_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&ctl.acc_full[i], 1); mbar_init(&ctl.acc_empty[i], G::SPLIT ? 8 : 4); }
-        mbar_init(&ctl.lr_full, 32);
-        mbar_init(&ctl.lr_empty, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl.lr_full[i], kLrThreads); mbar_init(&ctl.lr_empty[i], 1); }
         mbar_init(&ctl.drain, 1);
         ctl.wait.abort_flag = 0;
         ctl.wait.limit = p.wait_cycles;
@@ -299,7 +300,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                 const int ylr0 = y0 / R, xlr0 = x0 / R;
                 for (int g = 0; g < G::G && ok; ++g) {
                     for (int st = 0; st < p.nsteps; ++st) {
-                        if (!(ok = mbar_wait(&ctl.b_empty[s], ph ^ 1, wc))) break;
+                        if (!p.resident && !(ok = mbar_wait(&ctl.b_empty[s], ph ^ 1, wc))) break;
                         if (g == 0) {
                             if (!(ok = mbar_wait(&ctl.a_empty[st], (ti & 1) ^ 1, wc))) break;
                             const int nt = min(p.tps, p.ntaps - st * p.tps);
@@ -315,6 +316,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                             a_issued |= 1u << st;
                             a_parity = (a_parity & ~(1u << st)) | ((ti & 1) << st);
                         }
+                        if (p.resident && ti > 0) continue;      // resident weights: slot g * nsteps + st was filled for the first tile
                         if (lose_one && (st == 1 || p.nsteps == 1)) {
                             lose_one = false;                    // test hook: this stage never fills
                         } else {
@@ -360,7 +362,8 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                     if (!(ok = mbar_wait(&ctl.acc_empty[buf], ((pcount >> 1) & 1) ^ 1, wc))) break;
                     const uint32_t taddr = tmem_base + buf * 256u;
                     for (int st = 0; st < p.nsteps; ++st) {
-                        if (!(ok = mbar_wait(&ctl.b_full[s], ph, wc))) break;
+                        if (p.resident) s = g * p.nsteps + st;
+                        if ((!p.resident || ti == 0) && !(ok = mbar_wait(&ctl.b_full[s], p.resident ? 0u : ph, wc))) break;
                         if (g == 0 && !(ok = mbar_wait(&ctl.a_full[st], ti & 1, wc))) break;
                         tc_fence_after_sync();
                         const uint64_t bst = b_desc0 + (uint64_t)(((uint32_t)s * p.stage_bytes) >> 4);
@@ -373,9 +376,9 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                             mma_f16_ss(taddr, ad, bd, idesc, 1u);
                             mma_f16_ss(taddr, ad + (4096 >> 4), bd + ((2 * G::LBO_B) >> 4), idesc, 1u);
                         }
-                        mma_commit(&ctl.b_empty[s]);                 // the stage may be refilled once these MMAs have read it
+                        if (!p.resident) mma_commit(&ctl.b_empty[s]);   // the stage may be refilled once these MMAs have read it
                         if (g == G::G - 1) mma_commit(&ctl.a_empty[st]);   // and, after the tile's last pass, the feature taps
-                        if (++s == p.stages) { s = 0; ph ^= 1; }
+                        if (!p.resident && ++s == p.stages) { s = 0; ph ^= 1; }
                     }
                     if (ok) mma_commit(&ctl.acc_full[buf]);
                 }
@@ -385,15 +388,17 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             mbar_wait_drain(&ctl.drain, 0);
         }
         __syncwarp();
-    } else if (warp == kLrWarp) {
-        // ===== LR-window prefetch: the window of tile i + 1 travels while the epilogue works on tile i
+    } else if (warp == kLrWarp || warp == kLrWarp + 1) {
+        // ===== LR-window prefetch, two warps, two buffers: the windows of tiles i + 1 and i + 2 travel while the
+        // epilogue works on tile i (a window takes a microsecond or two to arrive from global memory)
         uint32_t ti = 0;
         for (int t = blockIdx.x; t < p.g.num_tiles; t += gridDim.x, ++ti) {
+            const uint32_t lb = ti & 1u;
             bool ok = true;
-            if (lane == 0) ok = mbar_wait_relaxed(&ctl.lr_empty, (ti & 1) ^ 1, wc);
+            if (lane == 0) ok = mbar_wait_relaxed(&ctl.lr_empty[lb], ((ti >> 1) & 1u) ^ 1u, wc);
             if (!__shfl_sync(0xffffffffu, (int)ok, 0)) break;
-            prefetch_lr_window<G::P>(p.g, p.lr, t, sL, lane, 32);
-            cp_async_mbar_arrive_noinc(&ctl.lr_full);
+            prefetch_lr_window<G::P>(p.g, p.lr, t, sL + lb * l_tile, tid - kLrWarp * 32, kLrThreads);
+            cp_async_mbar_arrive_noinc(&ctl.lr_full[lb]);
         }
         cp_async_wait_all();
     } else if (warp >= 4) {
@@ -416,12 +421,13 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             LrWindow w;
             lr_window<G::P>(p.g, t, w);
             const int uh = w.rows + 2 * G::P;
-            ok = ok && mbar_wait_leader(&ctl.lr_full, ti & 1, wc, true);
+            const uint32_t lb = ti & 1u;
+            ok = ok && mbar_wait_leader(&ctl.lr_full[lb], (ti >> 1) & 1u, wc, true);
             ok = named_barrier_and(1, kEpiThreads, ok);      // LR window landed, previous tile left by every thread
             if (!ok) break;
-            if (v_lane < v_lanes) vertical_pass(p.g, w, uh, G::P, sL, sV, v_i4, v_lane, v_lanes);
+            if (v_lane < v_lanes) vertical_pass(p.g, w, uh, G::P, sL + lb * l_tile, sV, v_i4, v_lane, v_lanes);
             named_barrier_sync(1, kEpiThreads);
-            if (et == 0) mbar_arrive(&ctl.lr_empty);         // the LR window may be overwritten
+            if (et == 0) mbar_arrive(&ctl.lr_empty[lb]);     // this LR window may be overwritten
             if (h_lane < h_lanes) horizontal_pass<G::P>(p.g, ctl.wpad, w, uh, sV, sU, h_cg, h_lane, h_lanes);
             named_barrier_sync(1, kEpiThreads);              // the U tile is complete
             const bool in_x = w.x0 + R * xl < pb.W;
@@ -557,7 +563,7 @@ constexpr int kStaticReserve = 4096;   // static shared memory (control block) +
 
 struct Plan {
     bool ok = false;
-    int ntaps = 0, tps = 0, nsteps = 0, stages = 0, passes = 0;
+    int ntaps = 0, tps = 0, nsteps = 0, stages = 0, passes = 0, resident = 0;
     uint32_t stage_bytes = 0;
     size_t smem = 0;
 };
@@ -576,8 +582,9 @@ Plan make_plan_rk(const Problem& pb, const ProducerShape& ps)
     // (taps per step) depends on scale, k and the layer only, as the header promises
     Problem pb3 = pb;
     pb3.c = kMaxC;
+    const size_t geom_floats = plan_geom(g, pb3, G::TH, nullptr);
     const size_t fixed = 1024 /* alignment slack */ + 32 + (size_t)pl.ntaps * kTapBytes + kOnesBytes +
-                         plan_geom(g, pb3, G::TH, nullptr) * sizeof(float);
+                         (geom_floats + (size_t)kMaxC * g.trows * g.tcols /* second LR window */) * sizeof(float);
     const size_t per_cta = (size_t)di.smem_optin - kStaticReserve;
     // a step = the taps of one kernel row when two such stages fit, else a single tap
     for (int tps = ps.kc; tps >= 1; tps = (tps > 1 ? 1 : 0)) {
@@ -588,6 +595,8 @@ Plan make_plan_rk(const Problem& pb, const ProducerShape& ps)
         pl.ok = true;
         pl.tps = tps;
         pl.nsteps = (pl.ntaps + tps - 1) / tps;
+        // when every stage of a tile fits at once the weights stay in shared memory for the CTA's whole life
+        if (stages >= G::G * pl.nsteps) { stages = G::G * pl.nsteps; pl.resident = 1; }
         pl.stages = stages;
         pl.stage_bytes = stage_bytes;
         pl.smem = fixed + (size_t)stages * stage_bytes;
@@ -702,7 +711,7 @@ cudaError_t launch_producer_regress(const float* lr, const void* feat, const voi
     if (!prm.status) return cudaErrorUnknown;
     const int th = pb.r * (128 / (TW / pb.r));
     plan_geom(prm.g, pb, th, lr);
-    prm.kc = ps.kc; prm.ntaps = pl.ntaps; prm.tps = pl.tps; prm.nsteps = pl.nsteps; prm.stages = pl.stages;
+    prm.kc = ps.kc; prm.ntaps = pl.ntaps; prm.tps = pl.tps; prm.nsteps = pl.nsteps; prm.stages = pl.stages; prm.resident = pl.resident;
     prm.stage_bytes = pl.stage_bytes;
     prm.wait_cycles = wait_cycle_limit();
     prm.inject_lost_arrival = take_injected_lost_arrival() ? 1 : 0;
