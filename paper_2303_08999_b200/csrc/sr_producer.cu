@@ -167,66 +167,80 @@ template <> __device__ __forceinline__ void store_pixels<2, uint8_t>(uint8_t* ds
     *reinterpret_cast<uchar2*>(dst) = make_uchar2(to_out<uint8_t>(v[0]), to_out<uint8_t>(v[1]));
 }
 
-// One pass of one tile for one thread: the RG phase rows of pass g for the r x r block of this thread's LR pixel.
+// One phase row (RYL, compile-time) of one pass for one thread: the r pixels of one HR row of this thread's r x r block.
+// The tensor-memory loads of patch row a + 1 are issued before the arithmetic of row a, so their latency hides behind it.
 //   u_px:   the up-sampled tile at (channel 0, row 0, this block's first column); planes u_plane floats apart
 //   out_px: channel 0, first row of the tile, this block's first pixel; channels HW elements apart
-//   only_ryl: the one phase row of the pass this thread takes (split passes), or -1 for all of them
-template <int R, int K, typename OutT>
-__device__ __forceinline__ void epilogue_pass(const float* u_px, int u_plane, OutT* out_px, int64_t HW, int W, int C, int g,
-                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01, int only_ryl)
+template <int R, int K, typename OutT, int RYL>
+__device__ __forceinline__ void epilogue_row(const float* u_px, int u_plane, OutT* out_px, int64_t HW, int W, int C, int g,
+                                             uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01)
 {
     using G = PG<R, K>;
     constexpr int UWIN = R + K - 1;                 // neighbouring values of a patch row the r pixels share
     constexpr int UV = R == 4 ? 4 : 2;              // floats per vector load (16- or 8-byte aligned at r * xl)
     constexpr int NV = (UWIN + UV - 1) / UV;
+    const int yt = R * yl + g * G::RG + RYL;        // row inside the tile
+    float acc[kMaxC][R];
 #pragma unroll
-    for (int ryl = 0; ryl < G::RG; ++ryl) {
-        if (only_ryl >= 0 && ryl != only_ryl) continue;
-        const int yt = R * yl + g * G::RG + ryl;    // row inside the tile
-        float acc[kMaxC][R];
+    for (int ch = 0; ch < kMaxC; ++ch)
 #pragma unroll
-        for (int ch = 0; ch < kMaxC; ++ch)
+        for (int rx = 0; rx < R; ++rx) acc[ch][rx] = 0.f;
+    float f[2][G::FWP];
+    tmem_ld_natural<G::FWP>(taddr, (RYL * K) * G::FWP, f[0]);
 #pragma unroll
-            for (int rx = 0; rx < R; ++rx) acc[ch][rx] = 0.f;
+    for (int a = 0; a < K; ++a) {
+        tmem_ld_wait();
+        if (a + 1 < K) tmem_ld_natural<G::FWP>(taddr, (RYL * K + a + 1) * G::FWP, f[(a + 1) & 1]);
+        const float* fa = f[a & 1];
+        float u[kMaxC][NV * UV];
 #pragma unroll
-        for (int a = 0; a < K; ++a) {
-            float f[G::FWP];
-            tmem_ld_natural<G::FWP>(taddr, (ryl * K + a) * G::FWP, f);
-            tmem_ld_wait();
+        for (int ch = 0; ch < kMaxC; ++ch) {
+            if (ch < C) {
+                const float* urow = u_px + ch * u_plane + (yt + a) * G::UW;
 #pragma unroll
-            for (int ch = 0; ch < kMaxC; ++ch) {
-                if (ch < C) {
-                    const float* urow = u_px + ch * u_plane + (yt + a) * G::UW;
-                    float u[NV * UV];
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) {
-                        if constexpr (UV == 4) {
-                            const float4 t = *reinterpret_cast<const float4*>(urow + 4 * i);
-                            u[4 * i] = t.x; u[4 * i + 1] = t.y; u[4 * i + 2] = t.z; u[4 * i + 3] = t.w;
-                        } else {
-                            const float2 t = *reinterpret_cast<const float2*>(urow + 2 * i);
-                            u[2 * i] = t.x; u[2 * i + 1] = t.y;
-                        }
+                for (int i = 0; i < NV; ++i) {
+                    if constexpr (UV == 4) {
+                        const float4 t = *reinterpret_cast<const float4*>(urow + 4 * i);
+                        u[ch][4 * i] = t.x; u[ch][4 * i + 1] = t.y; u[ch][4 * i + 2] = t.z; u[ch][4 * i + 3] = t.w;
+                    } else {
+                        const float2 t = *reinterpret_cast<const float2*>(urow + 2 * i);
+                        u[ch][2 * i] = t.x; u[ch][2 * i + 1] = t.y;
                     }
-#pragma unroll
-                    for (int rx = 0; rx < R; ++rx)
-#pragma unroll
-                        for (int b = 0; b < K; ++b) acc[ch][rx] = fmaf(f[rx * K + b], u[rx + b], acc[ch][rx]);
                 }
             }
         }
-        if (in_x && yt < rows_valid) {
+        // tap by tap across the r x c accumulators, so that consecutive multiply-adds are independent
 #pragma unroll
-            for (int ch = 0; ch < kMaxC; ++ch) {
+        for (int b = 0; b < K; ++b)
+#pragma unroll
+            for (int ch = 0; ch < kMaxC; ++ch)
                 if (ch < C) {
-                    if (clamp01) {
 #pragma unroll
-                        for (int rx = 0; rx < R; ++rx) acc[ch][rx] = fminf(fmaxf(acc[ch][rx], 0.f), 1.f);
-                    }
-                    store_pixels<R, OutT>(out_px + ch * HW + (int64_t)yt * W, acc[ch]);
+                    for (int rx = 0; rx < R; ++rx) acc[ch][rx] = fmaf(fa[rx * K + b], u[ch][rx + b], acc[ch][rx]);
                 }
+    }
+    if (in_x && yt < rows_valid) {
+#pragma unroll
+        for (int ch = 0; ch < kMaxC; ++ch) {
+            if (ch < C) {
+                if (clamp01) {
+#pragma unroll
+                    for (int rx = 0; rx < R; ++rx) acc[ch][rx] = fminf(fmaxf(acc[ch][rx], 0.f), 1.f);
+                }
+                store_pixels<R, OutT>(out_px + ch * HW + (int64_t)yt * W, acc[ch]);
             }
         }
+    }
+}
+
+// One pass of one tile for one thread: the RG phase rows of pass g, or only row `only_ryl` of them (split passes).
+template <int R, int K, typename OutT>
+__device__ __forceinline__ void epilogue_pass(const float* u_px, int u_plane, OutT* out_px, int64_t HW, int W, int C, int g,
+                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01, int only_ryl)
+{
+    if (only_ryl != 1) epilogue_row<R, K, OutT, 0>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
+    if constexpr (PG<R, K>::RG == 2) {
+        if (only_ryl != 0) epilogue_row<R, K, OutT, 1>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
     }
 }
 
