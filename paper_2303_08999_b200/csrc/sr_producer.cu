@@ -24,8 +24,8 @@
 // vector loads) and accumulates r x c outputs; r consecutive output pixels leave as one vector store. Two groups of four
 // warps take alternate passes. The up-sampled tile is built per tile by the epilogue warps (stage 1, Section II-A;
 // shared code with the other regression kernels).
-// Warps: 0 producer (TMA + bulk copies, one thread), 1 MMA issuer (one thread; owns tensor memory), 2-3 LR-window
-// prefetch (two windows ahead), 4-7 / 8-11 epilogue groups. One CTA per SM (512 TMEM columns), persistent over tiles.
+// Warps: 0 weight stages (bulk copies, one thread), 1 MMA issuer (one thread; owns tensor memory), 2 LR-window
+// prefetch (two windows ahead), 3 feature taps (TMA boxes, one thread), 4-7 / 8-11 epilogue groups. One CTA per SM (512 TMEM columns), persistent over tiles.
 // Every wait is bounded; on expiry the CTA raises its abort flag, sets the device status word, drains and returns.
 #include "sr_ptx.cuh"
 #include "sr_producer.cuh"
@@ -43,7 +43,7 @@ constexpr int kTapBytes = 128 * kCin * 2;   // one tap of the A operand: 128 pix
 constexpr int kOnesBytes = 128 * 16 * 2;    // the constant A tile of the bias K-step
 constexpr int kUtilThreads = 128, kEpiThreads = 256, kThreads = kUtilThreads + kEpiThreads;
 constexpr int kMaxSteps = 9, kMaxStages = 4, kMaxC = 3;
-constexpr int kMmaWarp = 1, kLrWarp = 2, kLrThreads = 64;   // warps 2 and 3 prefetch LR windows
+constexpr int kMmaWarp = 1, kLrWarp = 2, kLrThreads = 32, kFeatWarp = 3;
 
 template <int R, int K> struct PG {
     static constexpr int kk = K * K, P = (K - 1) / 2;
@@ -300,36 +300,17 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
 
     // ---------------------------------------------------------------- roles
     if (warp == 0) {
-        // ===== producer: feature taps (TMA boxes) on the first pass of a tile, folded weights (bulk copies) on every step
+        // ===== weight stages: one bulk copy per step of every pass, through the ring (or once per CTA when resident)
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0, ti = 0;
             bool ok = true;
             int issued_b = 0;
-            uint32_t a_issued = 0, a_parity = 0;              // per step: a box was issued; parity of its phase
             bool lose_one = p.inject_lost_arrival != 0 && blockIdx.x == 0;
             for (int t = blockIdx.x; t < p.g.num_tiles && ok; t += gridDim.x, ++ti) {
-                int f, y0, x0, rows;
-                decode_tile(p.g, t, f, y0, x0, rows);
-                const int ylr0 = y0 / R, xlr0 = x0 / R;
                 for (int g = 0; g < G::G && ok; ++g) {
                     for (int st = 0; st < p.nsteps; ++st) {
                         if (!p.resident && !(ok = mbar_wait(&ctl.b_empty[s], ph ^ 1, wc))) break;
-                        if (g == 0) {
-                            if (!(ok = mbar_wait(&ctl.a_empty[st], (ti & 1) ^ 1, wc))) break;
-                            const int nt = min(p.tps, p.ntaps - st * p.tps);
-                            mbar_arrive_expect_tx(&ctl.a_full[st], (uint32_t)(nt * kTapBytes));
-                            for (int j = 0; j < nt; ++j) {
-                                const int tap = st * p.tps + j;
-                                const int dy = tap / p.kc, dx = tap - dy * p.kc;
-                                uint8_t* dst = sA + (size_t)tap * kTapBytes;
-#pragma unroll
-                                for (int kg = 0; kg < kCin / 8; ++kg)
-                                    tma_load_4d(dst + kg * 2048, &map_feat, &ctl.a_full[st], kg * 8, xlr0 + dx - pc, ylr0 + dy - pc, f);
-                            }
-                            a_issued |= 1u << st;
-                            a_parity = (a_parity & ~(1u << st)) | ((ti & 1) << st);
-                        }
                         if (p.resident && ti > 0) continue;      // resident weights: slot g * nsteps + st was filled for the first tile
                         if (lose_one && (st == 1 || p.nsteps == 1)) {
                             lose_one = false;                    // test hook: this stage never fills
@@ -353,9 +334,37 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                     if (--sj < 0) { sj += p.stages; pj ^= 1; }
                     mbar_wait_drain(&ctl.b_full[sj], pj);
                 }
+            }
+        }
+        __syncwarp();
+    } else if (warp == kFeatWarp) {
+        // ===== feature taps: TMA boxes of the tile's taps, step by step, as soon as the previous tile's MMAs have read them
+        if (lane == 0) {
+            uint32_t ti = 0, a_issued = 0, a_parity = 0;      // per step: a box was issued; parity of its phase
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.g.num_tiles && ok; t += gridDim.x, ++ti) {
+                int f, y0, x0, rows;
+                decode_tile(p.g, t, f, y0, x0, rows);
+                const int ylr0 = y0 / R, xlr0 = x0 / R;
+                for (int st = 0; st < p.nsteps; ++st) {
+                    if (!(ok = mbar_wait(&ctl.a_empty[st], (ti & 1) ^ 1, wc))) break;
+                    const int nt = min(p.tps, p.ntaps - st * p.tps);
+                    mbar_arrive_expect_tx(&ctl.a_full[st], (uint32_t)(nt * kTapBytes));
+                    for (int j = 0; j < nt; ++j) {
+                        const int tap = st * p.tps + j;
+                        const int dy = tap / p.kc, dx = tap - dy * p.kc;
+                        uint8_t* dst = sA + (size_t)tap * kTapBytes;
+#pragma unroll
+                        for (int kg = 0; kg < kCin / 8; ++kg)
+                            tma_load_4d(dst + kg * 2048, &map_feat, &ctl.a_full[st], kg * 8, xlr0 + dx - pc, ylr0 + dy - pc, f);
+                    }
+                    a_issued |= 1u << st;
+                    a_parity = (a_parity & ~(1u << st)) | ((ti & 1) << st);
+                }
+            }
+            if (!ok)                                          // wind-down: boxes in flight get a short, bounded time to land
                 for (int st = 0; st < p.nsteps; ++st)
                     if (a_issued & (1u << st)) mbar_wait_drain(&ctl.a_full[st], (a_parity >> st) & 1u);
-            }
         }
         __syncwarp();
     } else if (warp == kMmaWarp) {
@@ -402,8 +411,8 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             mbar_wait_drain(&ctl.drain, 0);
         }
         __syncwarp();
-    } else if (warp == kLrWarp || warp == kLrWarp + 1) {
-        // ===== LR-window prefetch, two warps, two buffers: the windows of tiles i + 1 and i + 2 travel while the
+    } else if (warp == kLrWarp) {
+        // ===== LR-window prefetch, two buffers: the windows of tiles i + 1 and i + 2 travel while the
         // epilogue works on tile i (a window takes a microsecond or two to arrive from global memory)
         uint32_t ti = 0;
         for (int t = blockIdx.x; t < p.g.num_tiles; t += gridDim.x, ++ti) {
