@@ -281,7 +281,7 @@ void sr_tune_reset(void);
  *          layout is private to the library and depends on d->scale, d->k, cin, kc (not on n, c, h, w, D)
  *   out    [n][c][H][W], 16-byte aligned; fp32, or binary16 / uint8 with SR_OUT_F16 / SR_OUT_U8
  * flags of sr_producer_regress: SR_CLAMP01, SR_UPSAMPLE_BILINEAR, SR_OUT_F16, SR_OUT_U8.
- * Supported: scale 2 or 4, k in {3, 5, 7}, c <= 3, cin = 32, kc in {1, 3}; anything else is SR_ERR_UNSUPPORTED (there
+ * Supported: scale 2, 3 or 4, k in {3, 5, 7} (k <= 5 at scale 3), c <= 3, cin = 32, kc in {1, 3}; anything else is SR_ERR_UNSUPPORTED (there
  * is no slower path behind this call) and sr_producer_folded_bytes returns 0.  The folded weights are rounded to
  * binary16 (the bias keeps about 22 bits), feature values must be finite; results agree with the fp64 definition
  * within the binary16 tolerance of the other calls.  Asynchronous on `stream`; device-side waits are bounded as in

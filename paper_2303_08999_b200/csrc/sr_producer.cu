@@ -9,8 +9,8 @@
 // atom subset with weights gamma (Section III-A, Eq. 6 / Eq. 9) folds the same way (the sum runs over the subset).
 // launch_producer_fold builds W' and b' once per (network, dictionary); launch_producer_regress is the per-frame kernel.
 //
-// The kernel is an implicit GEMM on the tensor cores: M = 128 LR pixels of a tile (TW / r columns x r rows, so the HR
-// tile is 128 x r^2 pixels), K = kc^2 taps x 32 feature channels, N = the folded filters of a group of phase rows.
+// The kernel is an implicit GEMM on the tensor cores: M = 128 LR pixels of a tile (128 / r columns x r rows, so the HR
+// tile is 128 x r^2 pixels; at r = 3, 42 x 3 LR pixels = 126 of the 128 rows and an HR tile of 126 x 9), K = kc^2 taps x 32 feature channels, N = the folded filters of a group of phase rows.
 //   A: one TMA box per tap and 8-channel group from the channels-last feature map [n][h][w][32] (binary16); boxes that
 //      reach outside the map read zeros, which is the convolution's zero padding. K-major, no swizzle.
 //   B: W' as binary16, pre-arranged by the fold in the K-major core-matrix order the MMA reads, streamed from L2 by
@@ -47,21 +47,26 @@ constexpr int kMmaWarp = 1, kLrWarp = 2, kLrThreads = 32, kFeatWarp = 3;
 
 template <int R, int K> struct PG {
     static constexpr int kk = K * K, P = (K - 1) / 2;
-    static constexpr int TLW = TW / R;                 // LR columns of a tile
+    static constexpr int TWD = R == 3 ? 126 : TW;      // HR columns of a tile (a multiple of r)
+    static constexpr int TLW = TWD / R;                // LR columns of a tile
     static constexpr int TLH = 128 / TLW;              // LR rows of a tile
+    static constexpr int MPIX = TLW * TLH;             // LR pixels of a tile = rows of the MMA in use (128, or 126 at r = 3)
     static constexpr int TH = R * TLH;                 // HR rows of a tile
     static constexpr int FW = R * K;                   // taps of one patch row for the r pixels of an HR row of the block
     static constexpr int FWP = (FW + 3) & ~3;          // padded so that tensor-memory loads stay naturally aligned
-    static constexpr int RG = (R % 2 == 0 && 2 * K * FWP <= 256) ? 2 : 1;   // phase rows per pass (N <= 256)
+    static constexpr int RG = R == 3 ? (3 * K * FWP <= 256 ? 3 : 1)
+                                     : ((R % 2 == 0 && 2 * K * FWP <= 256) ? 2 : 1);   // phase rows per pass (N <= 256)
     static constexpr int G = R / RG;                   // passes per tile
-    static constexpr bool SPLIT = RG == 2;             // both epilogue groups work on every pass, one phase row each
+    static constexpr bool SPLIT = RG >= 2;             // both epilogue groups work on every pass: group e takes the phase
+                                                       // rows of the pass with ryl % 2 == e
     static constexpr int NCOL = RG * K * FWP;          // accumulator columns of a pass
     static constexpr int NG = (NCOL + 15) / 16 * 16;   // N of the MMA
-    static constexpr int UW = tile_uw(P), UW4 = UW / 4;
+    static constexpr int UW = tile_uw(P, TWD), UW4 = UW / 4;
+    static constexpr uint32_t TAP_TX = MPIX * kCin * 2;   // bytes the boxes of one tap bring
     static constexpr int LBO_B = NG * 16;              // bytes between the two 8-channel groups of a K-step of B
     static constexpr int BIAS_BYTES = 2 * LBO_B;       // one K-step
     static constexpr int TAP_B_BYTES = 4 * LBO_B;      // two K-steps (32 channels)
-    static_assert(TLW * TLH == 128 && (SPLIT || (G % 2) == 0) && NG <= 256, "tile or pass shape");
+    static_assert(MPIX <= 128 && MPIX > 96 && (SPLIT || (G % 2) == 0) && NG <= 256, "tile or pass shape");
     // accumulator column of tap (a, b) for pixel rx of phase row ryl
     __host__ __device__ static constexpr int col_of(int ryl, int a, int rx, int b) { return (ryl * K + a) * FWP + rx * K + b; }
 };
@@ -167,6 +172,19 @@ template <> __device__ __forceinline__ void store_pixels<2, uint8_t>(uint8_t* ds
     *reinterpret_cast<uchar2*>(dst) = make_uchar2(to_out<uint8_t>(v[0]), to_out<uint8_t>(v[1]));
 }
 
+template <> __device__ __forceinline__ void store_pixels<3, float>(float* dst, const float* v)
+{
+    dst[0] = v[0]; dst[1] = v[1]; dst[2] = v[2];
+}
+template <> __device__ __forceinline__ void store_pixels<3, __half>(__half* dst, const float* v)
+{
+    dst[0] = __float2half_rn(v[0]); dst[1] = __float2half_rn(v[1]); dst[2] = __float2half_rn(v[2]);
+}
+template <> __device__ __forceinline__ void store_pixels<3, uint8_t>(uint8_t* dst, const float* v)
+{
+    dst[0] = to_out<uint8_t>(v[0]); dst[1] = to_out<uint8_t>(v[1]); dst[2] = to_out<uint8_t>(v[2]);
+}
+
 // One phase row (RYL, compile-time) of one pass for one thread: the r pixels of one HR row of this thread's r x r block.
 // The tensor-memory loads of patch row a + 1 are issued before the arithmetic of row a, so their latency hides behind it.
 //   u_px:   the up-sampled tile at (channel 0, row 0, this block's first column); planes u_plane floats apart
@@ -177,7 +195,7 @@ __device__ __forceinline__ void epilogue_row(const float* u_px, int u_plane, Out
 {
     using G = PG<R, K>;
     constexpr int UWIN = R + K - 1;                 // neighbouring values of a patch row the r pixels share
-    constexpr int UV = R == 4 ? 4 : 2;              // floats per vector load (16- or 8-byte aligned at r * xl)
+    constexpr int UV = R == 4 ? 4 : (R == 2 ? 2 : 1);   // floats per load (16-, 8- or 4-byte aligned at r * xl)
     constexpr int NV = (UWIN + UV - 1) / UV;
     const int yt = R * yl + g * G::RG + RYL;        // row inside the tile
     float acc[kMaxC][R];
@@ -202,6 +220,8 @@ __device__ __forceinline__ void epilogue_row(const float* u_px, int u_plane, Out
                     if constexpr (UV == 4) {
                         const float4 t = *reinterpret_cast<const float4*>(urow + 4 * i);
                         u[ch][4 * i] = t.x; u[ch][4 * i + 1] = t.y; u[ch][4 * i + 2] = t.z; u[ch][4 * i + 3] = t.w;
+                    } else if constexpr (UV == 1) {
+                        u[ch][i] = urow[i];
                     } else {
                         const float2 t = *reinterpret_cast<const float2*>(urow + 2 * i);
                         u[ch][2 * i] = t.x; u[ch][2 * i + 1] = t.y;
@@ -233,14 +253,17 @@ __device__ __forceinline__ void epilogue_row(const float* u_px, int u_plane, Out
     }
 }
 
-// One pass of one tile for one thread: the RG phase rows of pass g, or only row `only_ryl` of them (split passes).
+// One pass of one tile for one thread: the RG phase rows of pass g (group < 0), or those with ryl % 2 == group (split passes).
 template <int R, int K, typename OutT>
 __device__ __forceinline__ void epilogue_pass(const float* u_px, int u_plane, OutT* out_px, int64_t HW, int W, int C, int g,
-                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01, int only_ryl)
+                                              uint32_t taddr, int yl, int rows_valid, bool in_x, bool clamp01, int group)
 {
-    if (only_ryl != 1) epilogue_row<R, K, OutT, 0>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
-    if constexpr (PG<R, K>::RG == 2) {
-        if (only_ryl != 0) epilogue_row<R, K, OutT, 1>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
+    if (group != 1) epilogue_row<R, K, OutT, 0>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
+    if constexpr (PG<R, K>::RG >= 2) {
+        if (group != 0) epilogue_row<R, K, OutT, 1>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
+    }
+    if constexpr (PG<R, K>::RG >= 3) {
+        if (group != 1) epilogue_row<R, K, OutT, 2>(u_px, u_plane, out_px, HW, W, C, g, taddr, yl, rows_valid, in_x, clamp01);
     }
 }
 
@@ -349,7 +372,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
                 for (int st = 0; st < p.nsteps; ++st) {
                     if (!(ok = mbar_wait(&ctl.a_empty[st], (ti & 1) ^ 1, wc))) break;
                     const int nt = min(p.tps, p.ntaps - st * p.tps);
-                    mbar_arrive_expect_tx(&ctl.a_full[st], (uint32_t)(nt * kTapBytes));
+                    mbar_arrive_expect_tx(&ctl.a_full[st], (uint32_t)nt * G::TAP_TX);
                     for (int j = 0; j < nt; ++j) {
                         const int tap = st * p.tps + j;
                         const int dy = tap / p.kc, dx = tap - dy * p.kc;
@@ -420,7 +443,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             bool ok = true;
             if (lane == 0) ok = mbar_wait_relaxed(&ctl.lr_empty[lb], ((ti >> 1) & 1u) ^ 1u, wc);
             if (!__shfl_sync(0xffffffffu, (int)ok, 0)) break;
-            prefetch_lr_window<G::P>(p.g, p.lr, t, sL + lb * l_tile, tid - kLrWarp * 32, kLrThreads);
+            prefetch_lr_window<G::P, G::TWD>(p.g, p.lr, t, sL + lb * l_tile, tid - kLrWarp * 32, kLrThreads);
             cp_async_mbar_arrive_noinc(&ctl.lr_full[lb]);
         }
         cp_async_wait_all();
@@ -429,7 +452,8 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
         const int e = (warp - 4) >> 2;                       // group: takes the passes with g % 2 == e
         const int quarter = warp & 3;                        // the TMEM lanes this warp may read: 32*quarter..+31
         const int m = quarter * 32 + lane;                   // LR pixel of the tile = TMEM lane
-        const int yl = m / G::TLW, xl = m - yl * G::TLW;
+        const bool lane_used = m < G::MPIX;                  // at r = 3 the last two rows of the MMA carry no pixel
+        const int yl = lane_used ? m / G::TLW : 0, xl = lane_used ? m - yl * G::TLW : 0;
         const int64_t HW = (int64_t)pb.H * pb.W;
         const bool clamp01 = (pb.flags & SR_CLAMP01) != 0;
         const uint32_t tmem_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -442,7 +466,7 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
         bool ok = true;
         for (int t = blockIdx.x; t < p.g.num_tiles; t += gridDim.x, ++ti) {
             LrWindow w;
-            lr_window<G::P>(p.g, t, w);
+            lr_window<G::P, G::TWD>(p.g, t, w);
             const int uh = w.rows + 2 * G::P;
             const uint32_t lb = ti & 1u;
             ok = ok && mbar_wait_leader(&ctl.lr_full[lb], (ti >> 1) & 1u, wc, true);
@@ -451,9 +475,9 @@ producer_regress_kernel(const __grid_constant__ CUtensorMap map_feat, const __gr
             if (v_lane < v_lanes) vertical_pass(p.g, w, uh, G::P, sL + lb * l_tile, sV, v_i4, v_lane, v_lanes);
             named_barrier_sync(1, kEpiThreads);
             if (et == 0) mbar_arrive(&ctl.lr_empty[lb]);     // this LR window may be overwritten
-            if (h_lane < h_lanes) horizontal_pass<G::P>(p.g, ctl.wpad, w, uh, sV, sU, h_cg, h_lane, h_lanes);
+            if (h_lane < h_lanes) horizontal_pass<G::P, G::TWD>(p.g, ctl.wpad, w, uh, sV, sU, h_cg, h_lane, h_lanes);
             named_barrier_sync(1, kEpiThreads);              // the U tile is complete
-            const bool in_x = w.x0 + R * xl < pb.W;
+            const bool in_x = lane_used && w.x0 + R * xl < pb.W;
             OutT* out_px = reinterpret_cast<OutT*>(p.out) + (int64_t)w.f * C * HW + (int64_t)w.y0 * pb.W + w.x0 + R * xl;
             // split passes: both groups take every pass (buffers alternate), group e the phase row e of it;
             // otherwise group e takes the passes with g % 2 == e, which always land in buffer e
@@ -605,7 +629,7 @@ Plan make_plan_rk(const Problem& pb, const ProducerShape& ps)
     // (taps per step) depends on scale, k and the layer only, as the header promises
     Problem pb3 = pb;
     pb3.c = kMaxC;
-    const size_t geom_floats = plan_geom(g, pb3, G::TH, nullptr);
+    const size_t geom_floats = plan_geom(g, pb3, G::TH, nullptr, G::TWD);
     const size_t fixed = 1024 /* alignment slack */ + 32 + (size_t)pl.ntaps * kTapBytes + kOnesBytes +
                          (geom_floats + (size_t)kMaxC * g.trows * g.tcols /* second LR window */) * sizeof(float);
     const size_t per_cta = (size_t)di.smem_optin - kStaticReserve;
@@ -635,6 +659,9 @@ Plan make_plan(const Problem& pb, const ProducerShape& ps)
         if (pb.k == 3) return make_plan_rk<4, 3>(pb, ps);
         if (pb.k == 5) return make_plan_rk<4, 5>(pb, ps);
         if (pb.k == 7) return make_plan_rk<4, 7>(pb, ps);
+    } else if (pb.r == 3) {
+        if (pb.k == 3) return make_plan_rk<3, 3>(pb, ps);
+        if (pb.k == 5) return make_plan_rk<3, 5>(pb, ps);
     } else if (pb.r == 2) {
         if (pb.k == 3) return make_plan_rk<2, 3>(pb, ps);
         if (pb.k == 5) return make_plan_rk<2, 5>(pb, ps);
@@ -715,6 +742,9 @@ cudaError_t launch_producer_fold(const float* wconv, const float* bias, const fl
         if (pb.k == 3) return fold_rk<4, 3>(out, fp, st);
         if (pb.k == 5) return fold_rk<4, 5>(out, fp, st);
         if (pb.k == 7) return fold_rk<4, 7>(out, fp, st);
+    } else if (pb.r == 3) {
+        if (pb.k == 3) return fold_rk<3, 3>(out, fp, st);
+        if (pb.k == 5) return fold_rk<3, 5>(out, fp, st);
     } else if (pb.r == 2) {
         if (pb.k == 3) return fold_rk<2, 3>(out, fp, st);
         if (pb.k == 5) return fold_rk<2, 5>(out, fp, st);
@@ -732,8 +762,8 @@ cudaError_t launch_producer_regress(const float* lr, const void* feat, const voi
     prm.lr = lr; prm.out = out; prm.folded = static_cast<const uint8_t*>(folded);
     prm.status = device_status_word();
     if (!prm.status) return cudaErrorUnknown;
-    const int th = pb.r * (128 / (TW / pb.r));
-    plan_geom(prm.g, pb, th, lr);
+    const int tw = pb.r == 3 ? 126 : TW, tlw = tw / pb.r, tlh = 128 / tlw;   // the tile shape of PG<R, K>
+    plan_geom(prm.g, pb, pb.r * tlh, lr, tw);
     prm.kc = ps.kc; prm.ntaps = pl.ntaps; prm.tps = pl.tps; prm.nsteps = pl.nsteps; prm.stages = pl.stages; prm.resident = pl.resident;
     prm.stage_bytes = pl.stage_bytes;
     prm.wait_cycles = wait_cycle_limit();
@@ -744,7 +774,7 @@ cudaError_t launch_producer_regress(const float* lr, const void* feat, const voi
     const cuuint64_t dims[4] = {(cuuint64_t)ps.cin, (cuuint64_t)pb.w, (cuuint64_t)pb.h, (cuuint64_t)pb.n};
     const cuuint64_t strides[3] = {(cuuint64_t)ps.cin * 2, (cuuint64_t)pb.w * ps.cin * 2, (cuuint64_t)pb.h * pb.w * ps.cin * 2};
     const cuuint32_t es[4] = {1, 1, 1, 1};
-    const cuuint32_t box[4] = {8, (cuuint32_t)(TW / pb.r), (cuuint32_t)(128 / (TW / pb.r)), 1};
+    const cuuint32_t box[4] = {8, (cuuint32_t)tlw, (cuuint32_t)tlh, 1};
     if (encode_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(feat), dims, strides, box, es,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -753,6 +783,9 @@ cudaError_t launch_producer_regress(const float* lr, const void* feat, const voi
         if (pb.k == 3) return launch_rk<4, 3>(map, prm, pl, st);
         if (pb.k == 5) return launch_rk<4, 5>(map, prm, pl, st);
         if (pb.k == 7) return launch_rk<4, 7>(map, prm, pl, st);
+    } else if (pb.r == 3) {
+        if (pb.k == 3) return launch_rk<3, 3>(map, prm, pl, st);
+        if (pb.k == 5) return launch_rk<3, 5>(map, prm, pl, st);
     } else if (pb.r == 2) {
         if (pb.k == 3) return launch_rk<2, 3>(map, prm, pl, st);
         if (pb.k == 5) return launch_rk<2, 5>(map, prm, pl, st);

@@ -9,7 +9,8 @@ struct ProducerShape {
     int cin, kc;
 };
 
-// True when the fused kernel runs the problem: scale 2 or 4, k in {3, 5, 7}, c <= 3, cin = 32, kc in {1, 3}.
+// True when the fused kernel runs the problem: scale 2, 3 or 4, k in {3, 5, 7} (k <= 5 at scale 3), c <= 3, cin = 32,
+// kc in {1, 3}.
 bool producer_supported(const Problem& pb, const ProducerShape& ps);
 
 // Bytes of the folded-weights block for the problem (0 when it is not supported).

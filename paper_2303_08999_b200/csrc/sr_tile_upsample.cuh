@@ -1,4 +1,5 @@
-// Up-sampled tile in shared memory, shared by the regression kernels that walk HR tiles of 128 x th pixels:
+// Up-sampled tile in shared memory, shared by the regression kernels that walk HR tiles of tw x th pixels (tw = 128
+// unless a kernel asks otherwise):
 // tile geometry, the LR window a tile needs, its asynchronous fetch, and the two separable passes (stage 1 of the
 // method, Section II-A; bicubic or bilinear taps come from the per-phase table in Problem).
 //   sL [c * nrows][tcols]   LR window (rows flattened as ch * nrows + j)
@@ -14,10 +15,11 @@
 namespace sr {
 namespace tile {
 
-constexpr int TW = 128;   // tile width in HR pixels
+constexpr int TW = 128;   // default tile width in HR pixels
 
 struct Geom {
     Problem pb;
+    int tw;               // tile width
     int th, uh;           // tile height, and th + 2 P (rows allocated for the U tile)
     int trows, tcols;     // LR rows / columns a tile can need (tcols a multiple of 4)
     int lr_vec;           // 1: LR rows are 16-byte aligned (16-byte copies for the inner part of the window)
@@ -27,13 +29,14 @@ struct Geom {
 };
 
 // U tile width for patch radius P: tile + halo, rounded up to 4 for 16-byte rows.
-__host__ __device__ constexpr int tile_uw(int P) { return (TW + 2 * P + 3) & ~3; }
+__host__ __device__ constexpr int tile_uw(int P, int tw = TW) { return (tw + 2 * P + 3) & ~3; }
 
 // Host side: fills th-dependent sizes; returns the floats the three buffers need.
-inline size_t plan_geom(Geom& g, const Problem& pb, int th, const float* lr)
+inline size_t plan_geom(Geom& g, const Problem& pb, int th, const float* lr, int tw = TW)
 {
-    const int P = (pb.k - 1) / 2, UW = tile_uw(P);
+    const int P = (pb.k - 1) / 2, UW = tile_uw(P, tw);
     g.pb = pb;
+    g.tw = tw;
     g.th = th;
     g.uh = th + 2 * P;
     g.trows = (g.uh - 1) / pb.r + 5;
@@ -42,7 +45,7 @@ inline size_t plan_geom(Geom& g, const Problem& pb, int th, const float* lr)
     g.r_magic = pb.r > 1 ? (uint32_t)((0x100000000ull + pb.r - 1) / pb.r) : 0u;
     const int tc4 = g.tcols / 4;
     g.tc4_magic = (uint32_t)((0x100000000ull + tc4 - 1) / tc4);
-    g.tiles_x = (pb.W + TW - 1) / TW;
+    g.tiles_x = (pb.W + tw - 1) / tw;
     g.tiles_y = (pb.H + th - 1) / th;
     g.num_tiles = g.tiles_x * g.tiles_y * pb.n;
     return (size_t)pb.c * g.uh * UW + (size_t)pb.c * g.uh * g.tcols + (size_t)pb.c * g.trows * g.tcols;
@@ -59,7 +62,7 @@ __device__ __forceinline__ void decode_tile(const Geom& p, int t, int& f, int& y
     const int ty = rest % p.tiles_y;
     f = rest / p.tiles_y;
     y0 = ty * p.th;
-    x0 = tx * TW;
+    x0 = tx * p.tw;
     rows = min(p.th, p.pb.H - y0);
 }
 
@@ -75,10 +78,10 @@ __device__ __forceinline__ int first_tap(const Geom& p, int Z, int& phase)
     return q + p.pb.ph.base[phase];
 }
 
-template <int P>
+template <int P, int TWD = TW>
 __device__ __forceinline__ void lr_window(const Geom& p, int t, LrWindow& g)
 {
-    constexpr int UW = tile_uw(P);
+    constexpr int UW = tile_uw(P, TWD);
     const Problem& pb = p.pb;
     decode_tile(p, t, g.f, g.y0, g.x0, g.rows);
     int ph;
@@ -102,13 +105,13 @@ __device__ __forceinline__ void cp_async_16(float* dst_smem, const float* src)
 // Fetches the LR window of tile t into dstL with asynchronous copies: 16 bytes where the four columns lie inside the
 // image and the row is aligned, single clamped elements at the borders. Thread `me` of `nthr`; the caller waits for
 // the copies (cp.async.wait_all or an mbarrier arrival).
-template <int P>
+template <int P, int TWD = TW>
 __device__ __forceinline__ void prefetch_lr_window(const Geom& p, const float* lr, int t, float* dstL, int me, int nthr)
 {
     const Problem& pb = p.pb;
     const int C = pb.c;
     LrWindow g;
-    lr_window<P>(p, t, g);
+    lr_window<P, TWD>(p, t, g);
     const int tc4 = p.tcols >> 2;
     const int total = C * g.nrows * tc4;
     for (int e = me; e < total; e += nthr) {
@@ -169,11 +172,11 @@ __device__ __forceinline__ void fill_wpad(const Problem& pb, float (*wpad)[12], 
 // neighbouring columns 4 cg .. 4 cg + 3 for the whole tile. Their first taps are at most three LR columns apart, so
 // the four outputs are one 4 x 7 matrix (taps shifted by each column's offset, zeros elsewhere; read from the
 // zero-padded weight table) times the seven values V[first .. first + 6]: seven shared loads per four outputs.
-template <int P>
+template <int P, int TWD = TW>
 __device__ __forceinline__ void horizontal_pass(const Geom& p, const float (*wpad)[12], const LrWindow& g, int uh, const float* sV,
                                                 float* sU, int cg, int row_lane, int row_lanes)
 {
-    constexpr int UW = tile_uw(P);
+    constexpr int UW = tile_uw(P, TWD);
     const Problem& pb = p.pb;
     float wm[4][7];
     int first = 0;

@@ -106,8 +106,8 @@ def test_validation_errors_come_back_before_any_launch(lib):
     assert lib.sr_producer_fold(FAKE, None, FAKE, FAKE, None, 99, FAKE, 16, ctypes.byref(d), 32, 3, None) == api.SR_ERR_SHAPE
     assert lib.sr_producer_regress(FAKE, None, FAKE, 16, FAKE, ctypes.byref(d), 32, 3, 0, None) == api.SR_ERR_NULL
     assert lib.sr_producer_regress(FAKE, FAKE, FAKE, 16, FAKE, ctypes.byref(d), 32, 3, api.SR_LUMA_ONLY, None) == api.SR_ERR_UNSUPPORTED
-    assert lib.sr_producer_regress(FAKE, FAKE, FAKE, 16, FAKE, ctypes.byref(_dims(scale=3)), 32, 3, 0, None) == api.SR_ERR_UNSUPPORTED
-    assert lib.sr_producer_folded_bytes(ctypes.byref(_dims(scale=3)), 32, 3) == 0
+    assert lib.sr_producer_regress(FAKE, FAKE, FAKE, 16, FAKE, ctypes.byref(_dims(scale=5)), 32, 3, 0, None) == api.SR_ERR_UNSUPPORTED
+    assert lib.sr_producer_folded_bytes(ctypes.byref(_dims(scale=5)), 32, 3) == 0
     assert lib.sr_producer_folded_bytes(ctypes.byref(d), 16, 3) == 0
 
 

@@ -28,7 +28,10 @@ CASES = [("r4_k5_ragged",        1, 3, 12, 40, 4, 8,  5, 3),
          ("r2_k5",               1, 3, 10, 70, 2, 16, 5, 3),
          ("r2_k3_one_channel",   1, 1, 5,  64, 2, 8,  3, 3),
          ("r2_k7",               2, 2, 6,  66, 2, 10, 7, 1),
-         ("r4_k5_many_tiles",    1, 3, 40, 72, 4, 72, 5, 3)]
+         ("r4_k5_many_tiles",    1, 3, 40, 72, 4, 72, 5, 3),
+         ("r3_k5_ragged",        1, 3, 11, 50, 3, 16, 5, 3),
+         ("r3_k3_two_frames",    2, 3, 7,  90, 3, 12, 3, 1),
+         ("r3_k5_one_channel",   1, 1, 20, 42, 3, 72, 5, 3)]
 
 
 def _make(case, seed=21):
@@ -95,10 +98,10 @@ def test_deterministic_and_unsupported_shapes():
     a = sr.sr_producer_regress(dev(lr), torch.from_numpy(feat).cuda(), folded, wl.scale, wl.k, wl.D, 3)
     b = sr.sr_producer_regress(dev(lr), torch.from_numpy(feat).cuda(), folded, wl.scale, wl.k, wl.D, 3)
     assert torch.equal(a, b)
-    w3 = sr_inputs.Workload("t", 1, 3, 8, 32, 3, D=8, k=5)
+    w3 = sr_inputs.Workload("t", 1, 3, 8, 32, 3, D=8, k=7)
     f3, wc3, b3 = sr_inputs.make_producer(w3, cin=32, kc=3)
-    with pytest.raises(sr.SrError):                          # scale 3 is not built
-        sr.sr_producer_fold(dev(wc3), dev(b3), dev(sr_inputs.make_dictionary(8, 5)), 3, 5)
+    with pytest.raises(sr.SrError):                          # 7 x 7 atoms at scale 3 are not built
+        sr.sr_producer_fold(dev(wc3), dev(b3), dev(sr_inputs.make_dictionary(8, 7)), 3, 7)
     f16c, wc16, b16 = sr_inputs.make_producer(wl, cin=16, kc=3)
     with pytest.raises(sr.SrError):                          # 16 feature channels are not built
         sr.sr_producer_fold(dev(wc16), dev(b16), dev(dict_), wl.scale, wl.k)
@@ -123,9 +126,10 @@ def test_a_lost_copy_times_out_and_the_next_call_is_correct():
     assert torch.equal(again, good)
 
 
-@pytest.mark.parametrize("name", ["cfg1", "cfg3"])
+@pytest.mark.parametrize("name", ["cfg1", "cfg3", "cfg4"])
 def test_full_size_whole_frame(name):
-    """The 1080p x4 frame of the benchmark and one frame of the 4K x2 batch, element by element over the whole output,
+    """The 1080p x4 frame of the benchmark, one frame of the 4K x2 batch and the x3 anchor of the sweep (360 x 640 LR),
+    element by element over the whole output,
     in the launch configuration bench.py times (signed, asymmetric dictionary)."""
     from dataclasses import replace
     wl = replace(sr_inputs.CONFIGS[name], n=1)
