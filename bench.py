@@ -121,7 +121,7 @@ def selection_network_ops_per_pixel(path: str, D: int, s: int):
 
 
 def fma_macs_per_pixel(wl, path: str):
-    """fp32 multiply-adds per HR pixel of the paths that run (or, by the survey's rule, are bounded) on the FMA pipe:
+    """fp32 multiply-adds per HR pixel of the paths that run on the FMA pipe, or are bounded by it because their atoms are too few for a tensor-core contraction:
     the small subset and compact forms (s k^2 + c k^2: assemble the filter from s atoms, then filter), and every
     regression with fp32 coefficients (general kernel: D k^2 + c k^2)."""
     kk = wl.k * wl.k

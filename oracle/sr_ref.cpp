@@ -29,7 +29,7 @@
  * responses built from the pinned dense regression, the LASSO against a library
  * solver and its optimality conditions, the re-fit against a library least-squares
  * solve, and the search against its stopping rules on hand-built problems.
- * The producer of Phi (last convolution + pixel-shuffle, the survey's producer-fusion row) is pinned in
+ * The producer of Phi (last convolution + pixel-shuffle of the coefficient network) is pinned in
  * tests/test_oracle_pins_producer.py against a library convolution and sub-pixel shuffle and against the pinned
  * dense regression fed with its output.
  * No function here is parity-unpinned.
@@ -168,7 +168,7 @@ void regress_pixel(const Dims& d, const float* dict, int natoms, const int* atom
     for (int q = 0; q < natoms; ++q)
         for (int j = 0; j < kk; ++j) F[j] += weights[q] * (double)dict[(int64_t)atoms[q] * kk + j];
     /*
-     * Luma-only regression (an I/O variant of this build, the usual practice of SR models that work on the Y channel;
+     * Luma-only regression (an I/O variant of this library, the usual practice of SR models that work on the Y channel;
      * not in the paper): the filter is applied to the luma Y = 0.299 R + 0.587 G + 0.114 B (BT.601) of the up-sampled
      * image, the two chroma differences keep their up-sampled values.  In RGB that is
      *     out_c = U_c + (F . B_Y - U_Y)       at the pixel, for c = R, G, B  (needs c = 3).
@@ -199,7 +199,7 @@ void regress_pixel(const Dims& d, const float* dict, int natoms, const int* atom
         }
         if (flags & REF_CLAMP01) acc = acc < 0.0 ? 0.0 : (acc > 1.0 ? 1.0 : acc);
         if (flags & REF_OUT_U8) {
-            /* 8-bit image output (an I/O variant of this build, not in the paper): the code of the value clamped to
+            /* 8-bit image output (an I/O variant of this library, not in the paper): the code of the value clamped to
              * [0,1] on the 255-step grid, nearest code, ties to the even one */
             const double v = acc < 0.0 ? 0.0 : (acc > 1.0 ? 1.0 : acc);
             acc = std::nearbyint(255.0 * v);
@@ -778,7 +778,8 @@ int sr_ref_selection_search(const double* G_in, const double* b_in, double hh, i
 
 /*
  * The producer of Phi (Section II-A, stage 2: LaparNet is a stack of fusion blocks, pixel-shuffle layers and
- * convolutions; only its last two layers are restated here, with seeded weights, as the survey's producer-fusion row).
+ * convolutions; only its last two layers are restated here, with seeded weights, for the call that fuses them with the
+ * regression).
  * The LR feature map feat[n][h][w][cin] (binary16, channels last) goes through one convolution with kc x kc taps,
  * zero padding kc/2, weights wconv[L r^2][cin][kc][kc] and bias[L r^2] (fp32), and a pixel-shuffle by r:
  *     Phi_l(Y, X) = conv[l r^2 + (Y mod r) r + (X mod r)](Y div r, X div r)
