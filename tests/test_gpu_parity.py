@@ -23,7 +23,8 @@ def _wl(n, c, h, w, r, D, k, dt):
 # ------------------------------------------------------------------ stage 1
 
 @pytest.mark.parametrize("n,c,h,w,r", [(1, 3, 64, 64, 2), (2, 3, 37, 53, 3), (1, 1, 5, 300, 4), (1, 2, 1, 1, 2),
-                                       (1, 3, 9, 7, 1), (1, 1, 6, 5, 8), (1, 4, 2, 3, 5)])
+                                       (1, 3, 9, 7, 1), (1, 1, 6, 5, 8), (1, 4, 2, 3, 5), (1, 3, 41, 35, 3), (2, 1, 9, 11, 6),
+                                       (1, 2, 13, 10, 5), (1, 1, 7, 9, 7)])
 def test_bicubic(n, c, h, w, r):
     lr = sr_inputs.make_lr(_wl(n, c, h, w, r, 1, 1, "f32"))
     got = host(sr.sr_bicubic_upsample(dev(lr), r))
