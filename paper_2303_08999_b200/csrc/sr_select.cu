@@ -158,6 +158,15 @@ select_pair_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
 // Needs 16-byte aligned planes (H * W a multiple of 8) and D KiB of shared memory.
 constexpr int kSelTilePixels = 512;
 
+// Byte permute with the full selector: bit 3 of a selector nibble replicates the sign bit of the selected byte instead
+// of copying it (the intrinsic only documents the low three bits).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
 __device__ __forceinline__ void sel_cp_async_16(uint32_t dst_smem, const void* src, uint32_t src_bytes)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
@@ -191,6 +200,12 @@ select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
 #pragma unroll
     for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1;
     int l0 = 0;
+    // Tags of four planes per register: byte j of tags[q] = 255 - (l0 + 4 q + j). A group moves them all down by S with
+    // one subtraction per register (no byte ever borrows: a tag is at least 255 - 199), instead of one per key.
+    uint32_t tags[S / 4];
+#pragma unroll
+    for (int q = 0; q < S / 4; ++q)
+        tags[q] = (255u - 4u * q) | ((254u - 4u * q) << 8) | ((253u - 4u * q) << 16) | ((252u - 4u * q) << 24);
     for (; l0 + S <= D; l0 += S) {                           // whole groups: no per-key guards
         uint32_t w[S];
 #pragma unroll
@@ -198,14 +213,18 @@ select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
         int ga[S], gb[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) {
-            const uint32_t tag = (uint32_t)(255 - (l0 + i)), m2 = w[i] & 0x7FFF7FFFu;
-            ga[i] = (int)__byte_perm(m2, tag, 0x5104);
-            gb[i] = (int)__byte_perm(m2, tag, 0x5324);
+            // key = (tag, magnitude low byte, magnitude high byte, 0): one byte permute per pixel out of (signs cleared,
+            // four tags); the top byte replicates the (cleared) sign bit of a magnitude byte, i.e. zero
+            const uint32_t m2 = w[i] & 0x7FFF7FFFu;
+            ga[i] = (int)prmt(m2, tags[i >> 2], 0x9100u | (uint32_t)(4 + (i & 3)));
+            gb[i] = (int)prmt(m2, tags[i >> 2], 0x9320u | (uint32_t)(4 + (i & 3)));
         }
         sort_desc<S>(ga);
         sort_desc<S>(gb);
         merge_top<S>(ta, ga);
         merge_top<S>(tb, gb);
+#pragma unroll
+        for (int q = 0; q < S / 4; ++q) tags[q] -= 0x01010101u * (uint32_t)S;
     }
     if (l0 < D) {                                            // last, partial group
         int ga[S], gb[S];
