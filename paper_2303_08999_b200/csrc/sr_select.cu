@@ -172,6 +172,56 @@ __device__ __forceinline__ void sel_cp_async_16(uint32_t dst_smem, const void* s
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
 }
 
+// ---- the same networks on keys held as fp32 numbers -------------------------------------------------------------------
+// A key (23 bits) is exactly representable in fp32, so a compare-exchange can run on either arithmetic pipe:
+//   ALU pipe:  hi = max(a, b), lo = min(a, b)                                    (2 operations, 64 lanes/clk/SM)
+//   FMA pipe:  d = a - b, s = a + b, hi = (s + |d|) / 2, lo = s - hi             (5 operations, 128 lanes/clk/SM)
+// every step of the second form is exact (integers below 2^24). The integer networks saturate the ALU pipe while the FMA
+// pipe idles. By pipe and issue-slot counts two exchanges in seven on the FMA pipe would be the balance; measured on the
+// 1080p frame the longer dependency chain of the second form matters as much: every fifth exchange, spread evenly, was
+// the fastest of eleven placements tried (118 us against 130 us with none; whole first layers on the FMA pipe: 131 us).
+__device__ __forceinline__ void cxf_alu(float& a, float& b)
+{
+    const float hi = fmaxf(a, b), lo = fminf(a, b);
+    a = hi;
+    b = lo;
+}
+__device__ __forceinline__ void cxf_fma(float& a, float& b)
+{
+    const float d = a - b, s = a + b;
+    const float hi = (s + fabsf(d)) * 0.5f;
+    b = s - hi;
+    a = hi;
+}
+// exchange number N of a network: which pipe takes it
+template <int N> __device__ __forceinline__ void cxf(float& a, float& b)
+{
+    if constexpr (N % 5 == 1) cxf_fma(a, b);
+    else cxf_alu(a, b);
+}
+
+__device__ __forceinline__ void sort8_desc_f(float* k)   // 19 exchanges
+{
+    cxf<0>(k[0], k[1]); cxf<1>(k[2], k[3]); cxf<2>(k[4], k[5]); cxf<3>(k[6], k[7]);
+    cxf<4>(k[0], k[2]); cxf<5>(k[1], k[3]); cxf<6>(k[4], k[6]); cxf<7>(k[5], k[7]);
+    cxf<8>(k[1], k[2]); cxf<9>(k[5], k[6]);
+    cxf<10>(k[0], k[4]); cxf<11>(k[1], k[5]); cxf<12>(k[2], k[6]); cxf<13>(k[3], k[7]);
+    cxf<14>(k[2], k[4]); cxf<15>(k[3], k[5]);
+    cxf<16>(k[1], k[2]); cxf<17>(k[3], k[4]); cxf<18>(k[5], k[6]);
+}
+
+// top[] (sorted) <- the 8 best of top[] and grp[] (grp sorted descending): 8 max, then a 12-exchange bitonic merge
+__device__ __forceinline__ void merge_top8_f(float* top, const float* grp)
+{
+#pragma unroll
+    for (int i = 0; i < 8; ++i) top[i] = fmaxf(top[i], grp[7 - i]);
+    cxf<19>(top[0], top[4]); cxf<20>(top[1], top[5]); cxf<21>(top[2], top[6]); cxf<22>(top[3], top[7]);
+    cxf<23>(top[0], top[2]); cxf<24>(top[1], top[3]); cxf<25>(top[4], top[6]); cxf<26>(top[5], top[7]);
+    cxf<27>(top[0], top[1]); cxf<28>(top[2], top[3]); cxf<29>(top[4], top[5]); cxf<30>(top[6], top[7]);
+}
+
+constexpr float kKeyMagic = 8388608.f;   // 2^23: the bits 0x4B000000 | key are the fp32 number 2^23 + key
+
 template <int S>
 __global__ void __launch_bounds__(256)
 select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
@@ -247,6 +297,89 @@ select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
     for (int q = 0; q < S; ++q) {
         if (q < s) {
             const int a = 255 - (ta[q] & 255), b = 255 - (tb[q] & 255);
+            const int64_t o = (f * s + q) * HW + pix;
+            *reinterpret_cast<uchar2*>(idx + o) = make_uchar2((unsigned char)a, (unsigned char)b);
+            if (sel) *reinterpret_cast<__half2*>(sel + o) = __halves2half2(th[a * kSelTilePixels], th[b * kSelTilePixels + 1]);
+        }
+    }
+}
+
+// The same tile kernel for lists of eight with the keys held as fp32 numbers, so that part of the compare-exchanges run
+// on the FMA pipe (see cxf). Three tags and the exponent byte 0x4B share a register: one prmt builds the bits of
+// 2^23 + key, one subtraction (FMA pipe) leaves the key.
+__global__ void __launch_bounds__(256)
+select_tile8f_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
+                     const __grid_constant__ Problem pb, int tiles_per_frame)
+{
+    constexpr int S = 8;
+    extern __shared__ __align__(16) uint8_t tile[];          // [D][512] binary16
+    const int64_t HW = (int64_t)pb.H * pb.W;
+    const int D = pb.D, s = pb.s, tid = threadIdx.x;
+    const int64_t f = blockIdx.x / tiles_per_frame;
+    const int64_t p0 = (int64_t)(blockIdx.x - f * tiles_per_frame) * kSelTilePixels;   // first pixel of the tile
+    const __half* cp = coef + f * D * HW + p0;
+    {
+        const uint32_t tile_s = (uint32_t)__cvta_generic_to_shared(tile);
+        const int chunk = tid & 63;                          // 16-byte chunk (8 pixels) of a plane's 1 KiB row
+        const uint32_t bytes = p0 + chunk * 8 < HW ? 16u : 0u;   // chunks beyond the frame are zero-filled
+        const __half* src = cp + (bytes ? chunk * 8 : 0);
+        for (int l = tid >> 6; l < D; l += 4)
+            sel_cp_async_16(tile_s + (uint32_t)l * 1024u + (uint32_t)chunk * 16u, src + (int64_t)l * HW, bytes);
+        asm volatile("cp.async.wait_all;" ::: "memory");
+    }
+    __syncthreads();
+    const int64_t pix = p0 + 2 * tid;
+    if (pix >= HW) return;
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(tile) + tid;   // + 256 words per plane
+    float ta[S], tb[S];
+#pragma unroll
+    for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1.f;
+    // byte j (j < 3) of tags[q] = 255 - (l0 + 3 q + j), byte 3 = 0x4B; a group moves the tags down by 8 with one
+    // subtraction per register (no byte ever borrows: a tag is at least 255 - 199)
+    uint32_t tags[3];
+#pragma unroll
+    for (int q = 0; q < 3; ++q) tags[q] = 0x4B000000u | (255u - 3u * q) | ((254u - 3u * q) << 8) | ((253u - 3u * q) << 16);
+    int l0 = 0;
+    for (; l0 + S <= D; l0 += S) {                           // whole groups: no per-key guards
+        uint32_t w[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) w[i] = wp[(l0 + i) * 256];
+        float ga[S], gb[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) {
+            // bits (tag, magnitude low byte, magnitude high byte, 0x4B) = the fp32 number 2^23 + key
+            const uint32_t m2 = w[i] & 0x7FFF7FFFu;
+            ga[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7100u | (uint32_t)(4 + i % 3))) - kKeyMagic;
+            gb[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7320u | (uint32_t)(4 + i % 3))) - kKeyMagic;
+        }
+        sort8_desc_f(ga);
+        sort8_desc_f(gb);
+        merge_top8_f(ta, ga);
+        merge_top8_f(tb, gb);
+#pragma unroll
+        for (int q = 0; q < 3; ++q) tags[q] -= 0x00080808u;
+    }
+    if (l0 < D) {                                            // last, partial group
+        float ga[S], gb[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) {
+            ga[i] = gb[i] = -1.f;
+            if (l0 + i < D) {
+                const uint32_t m2 = wp[(l0 + i) * 256] & 0x7FFF7FFFu;
+                ga[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7100u | (uint32_t)(4 + i % 3))) - kKeyMagic;
+                gb[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7320u | (uint32_t)(4 + i % 3))) - kKeyMagic;
+            }
+        }
+        sort8_desc_f(ga);
+        sort8_desc_f(gb);
+        merge_top8_f(ta, ga);
+        merge_top8_f(tb, gb);
+    }
+    const __half* th = reinterpret_cast<const __half*>(tile) + 2 * tid;
+#pragma unroll
+    for (int q = 0; q < S; ++q) {
+        if (q < s) {
+            const int a = 255 - (int)(__float_as_uint(ta[q] + kKeyMagic) & 255u), b = 255 - (int)(__float_as_uint(tb[q] + kKeyMagic) & 255u);
             const int64_t o = (f * s + q) * HW + pix;
             *reinterpret_cast<uchar2*>(idx + o) = make_uchar2((unsigned char)a, (unsigned char)b);
             if (sel) *reinterpret_cast<__half2*>(sel + o) = __halves2half2(th[a * kSelTilePixels], th[b * kSelTilePixels + 1]);
@@ -350,11 +483,11 @@ bool tile_path_ok(const void* coef, const Problem& pb)
            (HW + kSelTilePixels - 1) / kSelTilePixels * pb.n <= 0x7FFFFFFF;
 }
 
-template <int S>
+template <int S, bool FLOAT_KEYS = false>
 cudaError_t launch_tile_s(const __half* c, uint8_t* idx, __half* sl, const Problem& pb, cudaStream_t st)
 {
     const size_t smem = (size_t)pb.D * kSelTilePixels * sizeof(__half);
-    auto kern = select_tile_kernel<S>;
+    auto kern = FLOAT_KEYS ? select_tile8f_kernel : select_tile_kernel<S>;
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -374,7 +507,7 @@ cudaError_t launch_tile(const void* coef, uint8_t* idx, void* sel, const Problem
     const __half* c = (const __half*)coef;
     __half* sl = (__half*)sel;
     if (pb.s <= 4) return launch_tile_s<4>(c, idx, sl, pb, st);
-    if (pb.s <= 8) return launch_tile_s<8>(c, idx, sl, pb, st);
+    if (pb.s <= 8) return launch_tile_s<8, true>(c, idx, sl, pb, st);
     return launch_tile_s<16>(c, idx, sl, pb, st);
 }
 
