@@ -220,6 +220,59 @@ __device__ __forceinline__ void merge_top8_f(float* top, const float* grp)
     cxf<27>(top[0], top[1]); cxf<28>(top[2], top[3]); cxf<29>(top[4], top[5]); cxf<30>(top[6], top[7]);
 }
 
+// Lists of 4 and 16: the same split, the exchange number taken from its place in the network.
+__device__ __forceinline__ void sort4_desc_f(float* k)
+{
+    cxf<0>(k[0], k[1]); cxf<1>(k[2], k[3]);
+    cxf<2>(k[0], k[2]); cxf<3>(k[1], k[3]);
+    cxf<4>(k[1], k[2]);
+}
+__device__ __forceinline__ void merge_top4_f(float* top, const float* grp)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) top[i] = fmaxf(top[i], grp[3 - i]);
+    cxf<5>(top[0], top[2]); cxf<6>(top[1], top[3]);
+    cxf<7>(top[0], top[1]); cxf<8>(top[2], top[3]);
+}
+template <int BASE>
+__device__ __forceinline__ void bitonic16_desc_f(float* k)   // 32 exchanges, numbered from BASE
+{
+    cxf<BASE + 0>(k[0], k[8]); cxf<BASE + 1>(k[1], k[9]); cxf<BASE + 2>(k[2], k[10]); cxf<BASE + 3>(k[3], k[11]);
+    cxf<BASE + 4>(k[4], k[12]); cxf<BASE + 5>(k[5], k[13]); cxf<BASE + 6>(k[6], k[14]); cxf<BASE + 7>(k[7], k[15]);
+    cxf<BASE + 8>(k[0], k[4]); cxf<BASE + 9>(k[1], k[5]); cxf<BASE + 10>(k[2], k[6]); cxf<BASE + 11>(k[3], k[7]);
+    cxf<BASE + 12>(k[8], k[12]); cxf<BASE + 13>(k[9], k[13]); cxf<BASE + 14>(k[10], k[14]); cxf<BASE + 15>(k[11], k[15]);
+    cxf<BASE + 16>(k[0], k[2]); cxf<BASE + 17>(k[1], k[3]); cxf<BASE + 18>(k[4], k[6]); cxf<BASE + 19>(k[5], k[7]);
+    cxf<BASE + 20>(k[8], k[10]); cxf<BASE + 21>(k[9], k[11]); cxf<BASE + 22>(k[12], k[14]); cxf<BASE + 23>(k[13], k[15]);
+    cxf<BASE + 24>(k[0], k[1]); cxf<BASE + 25>(k[2], k[3]); cxf<BASE + 26>(k[4], k[5]); cxf<BASE + 27>(k[6], k[7]);
+    cxf<BASE + 28>(k[8], k[9]); cxf<BASE + 29>(k[10], k[11]); cxf<BASE + 30>(k[12], k[13]); cxf<BASE + 31>(k[14], k[15]);
+}
+__device__ __forceinline__ void sort16_desc_f(float* k)   // two sorted halves, then a bitonic merge
+{
+    sort8_desc_f(k);
+    sort8_desc_f(k + 8);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float t = k[8 + i]; k[8 + i] = k[15 - i]; k[15 - i] = t; }   // second half ascending
+    bitonic16_desc_f<19>(k);
+}
+__device__ __forceinline__ void merge_top16_f(float* top, const float* grp)
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) top[i] = fmaxf(top[i], grp[15 - i]);
+    bitonic16_desc_f<51>(top);
+}
+template <int S> __device__ __forceinline__ void sort_desc_f(float* k)
+{
+    if constexpr (S == 4) sort4_desc_f(k);
+    else if constexpr (S == 8) sort8_desc_f(k);
+    else sort16_desc_f(k);
+}
+template <int S> __device__ __forceinline__ void merge_top_f(float* top, const float* grp)
+{
+    if constexpr (S == 4) merge_top4_f(top, grp);
+    else if constexpr (S == 8) merge_top8_f(top, grp);
+    else merge_top16_f(top, grp);
+}
+
 constexpr float kKeyMagic = 8388608.f;   // 2^23: the bits 0x4B000000 | key are the fp32 number 2^23 + key
 
 template <int S>
@@ -304,14 +357,15 @@ select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
     }
 }
 
-// The same tile kernel for lists of eight with the keys held as fp32 numbers, so that part of the compare-exchanges run
+// The same tile kernel with the keys held as fp32 numbers, so that part of the compare-exchanges run
 // on the FMA pipe (see cxf). Three tags and the exponent byte 0x4B share a register: one prmt builds the bits of
 // 2^23 + key, one subtraction (FMA pipe) leaves the key.
+template <int S>
 __global__ void __launch_bounds__(256)
-select_tile8f_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
-                     const __grid_constant__ Problem pb, int tiles_per_frame)
+select_tilef_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
+                    const __grid_constant__ Problem pb, int tiles_per_frame)
 {
-    constexpr int S = 8;
+    constexpr int NT = (S + 2) / 3;                          // tag registers: three tags each
     extern __shared__ __align__(16) uint8_t tile[];          // [D][512] binary16
     const int64_t HW = (int64_t)pb.H * pb.W;
     const int D = pb.D, s = pb.s, tid = threadIdx.x;
@@ -334,11 +388,11 @@ select_tile8f_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx,
     float ta[S], tb[S];
 #pragma unroll
     for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1.f;
-    // byte j (j < 3) of tags[q] = 255 - (l0 + 3 q + j), byte 3 = 0x4B; a group moves the tags down by 8 with one
+    // byte j (j < 3) of tags[q] = 255 - (l0 + 3 q + j), byte 3 = 0x4B; a group moves the tags down by S with one
     // subtraction per register (no byte ever borrows: a tag is at least 255 - 199)
-    uint32_t tags[3];
+    uint32_t tags[NT];
 #pragma unroll
-    for (int q = 0; q < 3; ++q) tags[q] = 0x4B000000u | (255u - 3u * q) | ((254u - 3u * q) << 8) | ((253u - 3u * q) << 16);
+    for (int q = 0; q < NT; ++q) tags[q] = 0x4B000000u | (255u - 3u * q) | ((254u - 3u * q) << 8) | ((253u - 3u * q) << 16);
     int l0 = 0;
     for (; l0 + S <= D; l0 += S) {                           // whole groups: no per-key guards
         uint32_t w[S];
@@ -352,12 +406,12 @@ select_tile8f_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx,
             ga[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7100u | (uint32_t)(4 + i % 3))) - kKeyMagic;
             gb[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7320u | (uint32_t)(4 + i % 3))) - kKeyMagic;
         }
-        sort8_desc_f(ga);
-        sort8_desc_f(gb);
-        merge_top8_f(ta, ga);
-        merge_top8_f(tb, gb);
+        sort_desc_f<S>(ga);
+        sort_desc_f<S>(gb);
+        merge_top_f<S>(ta, ga);
+        merge_top_f<S>(tb, gb);
 #pragma unroll
-        for (int q = 0; q < 3; ++q) tags[q] -= 0x00080808u;
+        for (int q = 0; q < NT; ++q) tags[q] -= 0x00010101u * (uint32_t)S;
     }
     if (l0 < D) {                                            // last, partial group
         float ga[S], gb[S];
@@ -370,10 +424,10 @@ select_tile8f_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx,
                 gb[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7320u | (uint32_t)(4 + i % 3))) - kKeyMagic;
             }
         }
-        sort8_desc_f(ga);
-        sort8_desc_f(gb);
-        merge_top8_f(ta, ga);
-        merge_top8_f(tb, gb);
+        sort_desc_f<S>(ga);
+        sort_desc_f<S>(gb);
+        merge_top_f<S>(ta, ga);
+        merge_top_f<S>(tb, gb);
     }
     const __half* th = reinterpret_cast<const __half*>(tile) + 2 * tid;
 #pragma unroll
@@ -487,7 +541,7 @@ template <int S, bool FLOAT_KEYS = false>
 cudaError_t launch_tile_s(const __half* c, uint8_t* idx, __half* sl, const Problem& pb, cudaStream_t st)
 {
     const size_t smem = (size_t)pb.D * kSelTilePixels * sizeof(__half);
-    auto kern = FLOAT_KEYS ? select_tile8f_kernel : select_tile_kernel<S>;
+    auto kern = FLOAT_KEYS ? select_tilef_kernel<S> : select_tile_kernel<S>;
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -506,9 +560,9 @@ cudaError_t launch_tile(const void* coef, uint8_t* idx, void* sel, const Problem
 {
     const __half* c = (const __half*)coef;
     __half* sl = (__half*)sel;
-    if (pb.s <= 4) return launch_tile_s<4>(c, idx, sl, pb, st);
+    if (pb.s <= 4) return launch_tile_s<4, true>(c, idx, sl, pb, st);
     if (pb.s <= 8) return launch_tile_s<8, true>(c, idx, sl, pb, st);
-    return launch_tile_s<16>(c, idx, sl, pb, st);
+    return launch_tile_s<16, true>(c, idx, sl, pb, st);
 }
 
 cudaError_t launch_pair(const void* coef, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
