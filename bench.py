@@ -107,8 +107,10 @@ def selection_network_ops_per_pixel(path: str, D: int, s: int):
     (8 max + a 12-exchange bitonic merge for a list of 8; 8 max + 32 exchanges for a list of 16). The stand-alone kernel
     works on 32-bit keys, one pixel per lane operation; the fused kernel on packed binary16 pairs, two pixels per lane
     operation, plus 36 magnitude / logic and 40 address operations per 72 planes. These are the networks' own
-    operations: building the keys and the tails add about 45 % on the same pipe in the stand-alone kernel (ncu: ALU
-    pipe 84 % busy at 0.57 of this bound), instructions that are overhead to remove, not part of the bound."""
+    operations, all counted at the integer max/min rate: building the keys and the tails add to them on the same pipe
+    (overhead, not part of the bound), and the stand-alone kernel runs one compare-exchange in five on the FMA pipe
+    instead (five exact fp32 operations each), which is how it can come closer to this bound than the ALU pipe alone
+    would let it."""
     if s > 16 or path not in ("select", "fused"):
         return 0.0
     if path == "select":
