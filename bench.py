@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the dictionary-regression hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg0|cfg1|cfg2|cfg3|cfg4|producer]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg0|cfg1|cfg2|cfg3|cfg4|producer|extras]
 
 One step = one pass of the whole hot path over one frame batch of the workload (default: the
 1080p-output x4 frame, LR 3x270x480, D=72 atoms of 5x5, binary16 coefficients), i.e. six library
@@ -30,7 +30,8 @@ measured HBM bandwidth, its selection-network operations at the measured integer
 at the measured fp32 rate (both rates are measured at start-up by the library's probe kernels).
 `--workload producer` times the regression fused with the last layer of the coefficient network (sr_producer_regress, one
 call per step on the cfg1 frame, features [n][h][w][32] binary16, 3x3 convolution): its roofline is the folded
-convolution's tensor-core work against the measured dense bf16 rate.
+convolution's tensor-core work against the measured dense bf16 rate. `--workload extras` prints three more lines (output and
+up-sampling variants, the selection search, the tile-shape search); see run_extras.
 """
 from __future__ import annotations
 
@@ -672,6 +673,80 @@ def run_producer(wl, args, dist, rank, world, local_rank, steps: int, warmup: in
     }
 
 
+def run_extras(wl, args, peaks):
+    """`--workload extras`: the rows beyond the benchmark step, on the cfg1 frame, one JSON line each (CUDA events, median
+    of `--steps` launches after 3 warm-up launches, 256 MB written between launches to flush the L2):
+      variants   dense regression with binary16 / 8-bit output, bilinear up-sampling, luma-only
+      selection  Gram statistics of the selection search (every pixel; 100 000 sampled pixels) and Algorithm 1 on them
+      tune       the tile-shape search on three shapes: default launch shape against the best found"""
+    import numpy as np
+    import torch
+    import paper_2303_08999_b200 as sr
+    import sr_inputs
+    from dataclasses import replace
+
+    steps = max(5, min(args.steps, 50))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, reps=steps):
+        for _ in range(3):
+            fn()
+        ts = []
+        for i in range(reps):
+            flush.fill_(i & 255)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return statistics.median(ts), min(ts)
+
+    lr, dict_, coef = sr_inputs.make_inputs(wl)
+    dlr, ddi, dco = (torch.from_numpy(a).cuda() for a in (lr, dict_, coef))
+    r, k, s, D = wl.scale, wl.k, wl.s, wl.D
+    base = {"workload": f"{wl.name}: LR {wl.n}x{wl.c}x{wl.h}x{wl.w}, x{r}, D={D}, k={k}", "steps": steps, "unit": "us", "data": "synthetic"}
+    # ---- output and up-sampling variants of the dense call
+    out = {}
+    for name, fl in (("fp32 output", 0), ("binary16 output", sr.SR_OUT_F16), ("8-bit output", sr.SR_OUT_U8),
+                     ("bilinear up-sampling", sr.SR_UPSAMPLE_BILINEAR), ("luma-only (one-channel regression + chroma)", sr.SR_LUMA_ONLY)):
+        med, mn = timed(lambda: sr.sr_dict_regress_dense(dlr, dco, ddi, r, k, sr.SR_CLAMP01 | fl))
+        obytes = {0: 4, sr.SR_OUT_F16: 2, sr.SR_OUT_U8: 1}.get(fl, 4) * wl.c
+        by = (D * 2 + obytes + 4 * wl.c / r ** 2) * wl.npix
+        out[name] = {"median_us": med, "min_us": mn, "algorithmic_bytes": by, "frac_of_hbm": by / (med * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+    print(json.dumps(dict(base, extra="variants of sr_dict_regress_dense", results=out)), flush=True)
+    # ---- selection search: Gram statistics + Algorithm 1
+    S = np.arange(0, D, max(1, D // s), dtype=np.uint8)[:s]
+    gamma = np.linspace(0.75, 1.25, s).astype(np.float32)
+    target = sr.sr_dict_regress_selected(dlr, dco, torch.from_numpy(S).cuda(), torch.from_numpy(gamma).cuda(), ddi, r, k, s, sr.SR_IDX_GLOBAL)
+    target = (target + 0.01 * torch.randn(target.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(1))).contiguous()
+    samples = torch.arange(0, wl.npix, max(1, wl.npix // 100000), device="cuda", dtype=torch.int64)[:100000].contiguous()
+    macs_row = D * k * k + D * (D + 1) / 2 + D            # responses, upper triangle of z z^T, z h
+    res = {}
+    for name, smp, npx in (("every pixel", None, wl.npix), (f"{samples.numel()} sampled pixels", samples, samples.numel())):
+        med, mn = timed(lambda: sr.sr_selection_gram(dlr, dco, ddi, target, smp, r, k), reps=max(3, steps // 5))
+        macs = macs_row * npx * wl.c
+        res["gram, " + name] = {"median_us": med, "min_us": mn, "fp32_macs": macs, "frac_of_fma": macs / (med * 1e-6) / peaks["fma_ops"]}
+    G, b, hh = sr.sr_selection_gram(dlr, dco, ddi, target, samples, r, k)
+    t0 = time.perf_counter()
+    idx, gam, trace = sr.sr_selection_search(G, b, hh, samples.numel() * wl.c, s / D, 16.0 / D, 0.0, 1e-9)
+    torch.cuda.synchronize()
+    res["search (Algorithm 1, one warp, fp64)"] = {"wall_us": (time.perf_counter() - t0) * 1e6, "atoms_kept": int(idx.numel()),
+                                                   "steps": int(trace.shape[0]), "found_the_planted_subset": bool(np.array_equal(idx.cpu().numpy(), S))}
+    print(json.dumps(dict(base, extra="selection search (sr_selection_gram, sr_selection_search)", results=res)), flush=True)
+    # ---- tile-shape search
+    res = {}
+    for name, w2 in (("cfg1 dense", wl), ("cfg4 r2 D16 k7 dense", replace(sr_inputs.CONFIGS["cfg4"], scale=2, D=16, k=7)),
+                     ("cfg4 r3 D32 k5 dense", replace(sr_inputs.CONFIGS["cfg4"], scale=3, D=32, k=5))):
+        l2, d2, c2 = (torch.from_numpy(a).cuda() for a in sr_inputs.make_inputs(w2))
+        sr.sr_tune_reset()
+        res[name] = sr.sr_tune_dense(l2, c2, d2, w2.scale, w2.k, sr.SR_CLAMP01, reps=10)
+        S2 = torch.arange(0, w2.D, max(1, w2.D // 16), dtype=torch.uint8, device="cuda")[:16].contiguous()
+        if S2.numel() == 16:
+            res[name.replace("dense", "global subset s=16")] = sr.sr_tune_selected(l2, c2, S2, None, d2, w2.scale, w2.k, 16, sr.SR_CLAMP01 | sr.SR_IDX_GLOBAL, reps=10)
+        del l2, d2, c2
+    sr.sr_tune_reset()
+    print(json.dumps(dict(base, extra="tile-shape search (sr_tune_dense, sr_tune_selected): default launch shape against the best of the candidates", results=res)), flush=True)
+
+
 def load_tensor_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -707,7 +782,7 @@ def main():
     import sr_inputs
     from dataclasses import replace
     producer = args.workload == "producer"
-    if producer:
+    if producer or args.workload == "extras":
         wls = [sr_inputs.CONFIGS["cfg1"]]
     elif sweep:
         want = [w for w in args.points.split(",") if w]
@@ -735,6 +810,12 @@ def main():
     sr.load_library()
     peaks = measure_peaks(sr)
     default_line = args.workload in ("cfg1", "cfg2")
+    if args.workload == "extras":
+        if rank == 0:
+            run_extras(sr_inputs.CONFIGS["cfg1"], args, peaks)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     for wl in wls:
         if producer:
             line = run_producer(wl, args, dist, rank, world, local_rank, steps, warmup)

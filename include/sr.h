@@ -82,7 +82,10 @@ enum {
                                   the luma Y = 0.299 R + 0.587 G + 0.114 B of the up-sampled image and the chroma
                                   differences keep their up-sampled values:  out_ch = U_ch + (F . B_Y - U_Y)  at the
                                   pixel.  The common practice of SR models that predict on the Y channel; the paper
-                                  has no such variant.  Runs on the general fp32 kernel, whatever the shape.   */
+                                  has no such variant.  With fp32 output it is composed of the one-channel
+                                  regression of the luma frame (the fast kernels) and two small kernels, using
+                                  `out` itself as scratch; with binary16 / 8-bit output it runs on the general
+                                  fp32 kernel.                                                                  */
 };
 
 enum {

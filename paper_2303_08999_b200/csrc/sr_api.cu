@@ -211,8 +211,40 @@ static cudaError_t run_kernel(const TuneChoice& c, const RegressArgs& a)
     }
 }
 
+static cudaError_t run_regress(const RegressArgs& a);
+
+// SR_LUMA_ONLY with fp32 output: the one-channel regression of the frame's luma by the ordinary kernels, then the chroma
+// put back (sr_luma.cu). Planes 0 and 1 of the frame's own output serve as scratch.
+static cudaError_t run_regress_luma(const RegressArgs& a)
+{
+    const Problem& pb = a.pb;
+    const int64_t HW = (int64_t)pb.H * pb.W, hw = (int64_t)pb.h * pb.w;
+    const bool compact = a.mode == kModeCompact || (a.mode == kModeGlobal && (pb.flags & SR_COEF_COMPACT));
+    const int64_t coef_frame = (int64_t)(compact ? pb.s : pb.D) * HW * (a.coef_dtype == SR_F16 ? 2 : 4);
+    const bool idx_planes = a.idx && a.mode != kModeGlobal;
+    for (int f = 0; f < pb.n; ++f) {
+        const float* lr_f = a.lr + (int64_t)f * 3 * hw;
+        float* out_f = a.out + (int64_t)f * 3 * HW;
+        float* ylr = out_f + HW;
+        cudaError_t e = launch_luma_lr(lr_f, ylr, pb, a.st);
+        if (e != cudaSuccess) return e;
+        RegressArgs b = a;
+        b.lr = ylr;
+        b.out = out_f;
+        b.coef = static_cast<const uint8_t*>(a.coef) + (int64_t)f * coef_frame;
+        if (idx_planes) b.idx = a.idx + (int64_t)f * pb.s * HW;
+        b.pb.n = 1;
+        b.pb.c = 1;
+        b.pb.flags &= ~(uint32_t)(SR_LUMA_ONLY | SR_CLAMP01);
+        if ((e = run_regress(b)) != cudaSuccess) return e;
+        if ((e = launch_luma_combine(lr_f, out_f, pb, a.st)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 static cudaError_t run_regress(const RegressArgs& a)
 {
+    if ((a.pb.flags & SR_LUMA_ONLY) && !(a.pb.flags & (SR_OUT_F16 | SR_OUT_U8))) return run_regress_luma(a);
     TuneChoice c;
     if (tune_lookup(tune_key(a.mode, a.coef_dtype, a.pb), c) && kernel_supported(c.kernel, a)) return run_kernel(c, a);
     c = TuneChoice{};

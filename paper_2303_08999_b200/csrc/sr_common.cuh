@@ -62,6 +62,9 @@ cudaError_t launch_bicubic(const float* lr, float* hr, const Problem& pb, cudaSt
 cudaError_t launch_regress_fma(int mode, const float* lr, const void* coef, int coef_dtype, const uint8_t* idx,
                                const float* gamma, const float* dict, float* out, const Problem& pb, cudaStream_t st);
 cudaError_t launch_select(const void* coef, int coef_dtype, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st);
+// Steps 1 and 3 of the composed luma-only regression (sr_luma.cu), one frame at a time.
+cudaError_t launch_luma_lr(const float* lr_frame, float* ylr, const Problem& pb, cudaStream_t st);
+cudaError_t launch_luma_combine(const float* lr_frame, float* out_frame, const Problem& pb, cudaStream_t st);
 
 // ---- device helpers ------------------------------------------------------------------------------------------------
 

@@ -59,8 +59,11 @@ def test_output_types_and_chroma():
     f32 = sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5, LU)
     f16 = sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5, LU | sr.SR_OUT_F16)
     u8 = sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5, LU | sr.SR_OUT_U8)
-    assert f16.dtype == torch.float16 and torch.equal(f16, f32.to(torch.float16))
-    assert u8.dtype == torch.uint8 and torch.equal(u8, torch.round(torch.clamp(f32, 0, 1) * 255).to(torch.uint8))
+    # the fp32 form is composed of the fast one-channel regression and two small kernels, the other output types run on
+    # the general kernel: same definition, different rounding order
+    assert f16.dtype == torch.float16 and float((f16.float() - f32).abs().max()) <= 2 * TOL_F16 + 1e-3
+    codes = torch.round(torch.clamp(f32, 0, 1) * 255).to(torch.int16)
+    assert u8.dtype == torch.uint8 and int((u8.to(torch.int16) - codes).abs().max()) <= 1
     # without a clamp every channel moves by the same amount: differences between channels are those of stage 1
     U = sr.sr_bicubic_upsample(dlr, 2)
     assert float(((f32[:, 0] - f32[:, 1]) - (U[:, 0] - U[:, 1])).abs().max()) <= 1e-6
