@@ -240,7 +240,7 @@ int sr_device_status(void* stream, int* out_status);
  * Tile-shape search (Section III-B, restated for this library).  The paper prunes the space of thread-block shapes
  * of its filtering kernel with resource constraints (Eq. 11-12) and searches the rest by measured latency.  Here the
  * tunable shape of a regression launch is: which kernel takes it (first or second tensor-core layout, the FMA-pipe
- * subset kernel), the tile height, and the rows per pipeline step; the legal set follows from the shared memory per
+ * subset kernel, the FMA-pipe gather kernel for index + value planes), the tile height, and the rows per pipeline step; the legal set follows from the shared memory per
  * thread block, the tensor-memory columns and the stage count, and is small enough to time exhaustively.
  * sr_tune_dense / sr_tune_selected take the arguments of the call they tune plus `reps`, run every legal shape
  * (one warm-up launch, then `reps` timed launches between two CUDA events) on the caller's own buffers, and record the
@@ -251,8 +251,9 @@ int sr_device_status(void* stream, int* out_status);
  * every shape.  *result (may be NULL) receives the choice.  sr_tune_reset forgets every recorded shape.
  */
 typedef struct sr_tune_result {
-    int32_t kernel;        /* 0 general FMA kernel, 1 first tensor-core layout, 2 second tensor-core layout, 3 subset kernel */
-    int32_t tile_rows;     /* tile height (kernels 2 and 3; 0 otherwise)                                               */
+    int32_t kernel;        /* 0 general FMA kernel, 1 first tensor-core layout, 2 second tensor-core layout, 3 subset
+                              kernel, 4 gather kernel for index + value planes                                         */
+    int32_t tile_rows;     /* tile height (kernels 2, 3 and 4; 0 otherwise)                                            */
     int32_t rows_per_step; /* tile rows per pipeline step (kernel 2; 0 otherwise)                                      */
     int32_t candidates;    /* launch shapes that were legal and timed                                                   */
     float best_us;         /* time per launch of the recorded shape                                                     */
@@ -322,6 +323,14 @@ int64_t sr_set_wait_limit(int64_t cycles);
  * as described above.  0 disarms.  Returns SR_OK, or SR_ERR_SHAPE for a negative count.  The paper has no counterpart.
  */
 int sr_test_lose_arrival(int launches);
+
+/*
+ * Test hook: regression calls that follow are run by kernel `kernel` (the numbering of sr_tune_result.kernel)
+ * whenever that kernel supports the call, instead of the one the host rules or the tuning table pick; -1 restores
+ * the rules.  Lets a test compare two kernels that serve the same call.  Returns SR_OK, or SR_ERR_SHAPE for a number
+ * that names no kernel.  The paper has no counterpart.
+ */
+int sr_test_force_kernel(int kernel);
 
 /*
  * Number of kernels this library has launched in this process so far (all devices, all streams).

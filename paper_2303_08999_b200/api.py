@@ -20,7 +20,7 @@ SR_CLAMP01, SR_IDX_GLOBAL, SR_COEF_COMPACT, SR_UPSAMPLE_BILINEAR, SR_OUT_F16, SR
 SR_OK, SR_ERR_NULL, SR_ERR_SHAPE, SR_ERR_UNSUPPORTED, SR_ERR_ALIGN, SR_ERR_CUDA, SR_ERR_TIMEOUT, SR_ERR_TOO_LARGE = range(8)
 
 EXPORTS = ("sr_bicubic_upsample", "sr_bilinear_upsample", "sr_dict_regress_dense", "sr_dict_select", "sr_dict_regress_selected",
-           "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival",
+           "sr_status_string", "sr_device_status", "sr_launch_count", "sr_set_wait_limit", "sr_test_lose_arrival", "sr_test_force_kernel",
            "sr_selection_gram", "sr_selection_gram_scratch_bytes", "sr_selection_search", "sr_selection_search_scratch_bytes",
            "sr_selection_gram_static", "sr_probe_rate", "sr_tune_dense", "sr_tune_selected", "sr_tune_reset",
            "sr_producer_folded_bytes", "sr_producer_fold", "sr_producer_regress")
@@ -72,6 +72,7 @@ def load_library() -> ctypes.CDLL:
         lib.sr_set_wait_limit.argtypes = [ctypes.c_int64]
         lib.sr_set_wait_limit.restype = ctypes.c_int64
         lib.sr_test_lose_arrival.argtypes = [i32]
+        lib.sr_test_force_kernel.argtypes = [i32]
         i64, f64, sz = ctypes.c_int64, ctypes.c_double, ctypes.c_size_t
         lib.sr_selection_gram_scratch_bytes.argtypes = [dp]
         lib.sr_selection_gram_scratch_bytes.restype = sz
@@ -233,6 +234,15 @@ def sr_test_lose_arrival(launches: int) -> None:
     _check(load_library().sr_test_lose_arrival(int(launches)), "sr_test_lose_arrival")
 
 
+KERNEL_NAMES = {0: "general", 1: "first tensor-core layout", 2: "second tensor-core layout", 3: "subset (FMA pipe)",
+                4: "gather (FMA pipe)"}
+
+
+def sr_test_force_kernel(kernel: int) -> None:
+    """Test hook: later regression calls run on kernel `kernel` (a key of KERNEL_NAMES) where it supports them; -1 = host rules."""
+    _check(load_library().sr_test_force_kernel(int(kernel)), "sr_test_force_kernel")
+
+
 def sr_selection_gram(lr, coef, dict_, target, samples, scale: int, k: int, flags: int = 0):
     """Gram statistics of the dictionary selection search: returns (G [D][D], b [D], hh [1]) as float64 CUDA tensors.
     `samples`: int64 CUDA tensor of flat [n][H][W] pixel indices, or None for every pixel."""
@@ -333,8 +343,7 @@ def sr_producer_regress(lr, feat, folded, scale: int, k: int, D: int, kc: int, f
 
 
 def _tune_dict(res: sr_tune_result) -> dict:
-    names = {0: "general", 1: "first tensor-core layout", 2: "second tensor-core layout", 3: "subset (FMA pipe)"}
-    return {"kernel": names.get(res.kernel, str(res.kernel)), "tile_rows": res.tile_rows, "rows_per_step": res.rows_per_step,
+    return {"kernel": KERNEL_NAMES.get(res.kernel, str(res.kernel)), "tile_rows": res.tile_rows, "rows_per_step": res.rows_per_step,
             "candidates": res.candidates, "best_us": res.best_us, "default_us": res.default_us}
 
 

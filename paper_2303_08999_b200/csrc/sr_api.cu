@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "sr_common.cuh"
+#include "sr_regress_listed.cuh"
 #include "sr_regress_subset.cuh"
 #include "sr_producer.cuh"
 #include "sr_regress_tc.cuh"
@@ -37,6 +38,7 @@ int* device_status_word()
 
 static std::atomic<long long> g_wait_limit{1ll << 31};
 static std::atomic<int> g_lose_arrival{0};
+static std::atomic<int> g_force_kernel{-1};
 
 long long wait_cycle_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
 
@@ -124,6 +126,20 @@ static bool bad_out_flags(uint32_t flags, const sr_dims* d)
 // on the 1080p sweep points (dense, D = 16 / 32 / 72 / 128; k = 3 / 5 / 7).
 static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 || (pb.k == 7 && pb.D <= 32); }
 
+// Which kernel takes a launch from index + value planes when both could. The gather kernel (sr_regress_listed.cu) pays
+// s * ceil(k^2 / 4) 16-byte shared-memory gathers per pixel and nothing per atom of the dictionary; the first
+// tensor-core layout pays for clearing and filling a stage row of D coefficients per pixel and little per listed atom.
+// Measured on the 1080p sweep points and the 4K x2 batch (D = 16 / 32 / 72 / 128; k = 3 / 5 / 7; s = 4 / 8 / 16): the
+// gather kernel is 1.0 - 3.4 times faster wherever one of these holds, and up to two times slower at the far end
+// (k = 7, s = 16).
+static bool compact_prefers_listed(const Problem& pb)
+{
+    const int gathers = pb.s * ((pb.k * pb.k + 3) / 4);
+    if (pb.D > 96 || gathers <= 28) return true;
+    if (pb.D >= 64) return gathers <= 52 || (gathers <= 56 && pb.r == 2);
+    return false;
+}
+
 // ---- which kernel runs a regression, and in which launch shape ----------------------------------------------------------
 //
 // Every regression call goes through run_regress. Without an entry in the tuning table it takes the kernel and shape
@@ -131,12 +147,12 @@ static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 |
 // the fastest for that problem shape (the block-shape search of Section III-B, restated for this library: the legal
 // set comes from shared-memory, tensor-memory and stage-count constraints instead of register-file and warp-scheduler
 // limits, and it is small enough to be timed exhaustively instead of by Bayesian optimisation).
-enum RegressKernel { kKernelGeneral = 0, kKernelFirstLayout = 1, kKernelSecondLayout = 2, kKernelSubset = 3 };
+enum RegressKernel { kKernelGeneral = 0, kKernelFirstLayout = 1, kKernelSecondLayout = 2, kKernelSubset = 3, kKernelListed = 4 };
 
 struct TuneChoice {
     int kernel = -1;      // -1: host rules
     TcTuning tc;          // second layout: tile height and rows per pipeline step
-    int sub_th = 0;       // subset kernel: tile height
+    int sub_th = 0;       // subset and listed kernels: tile height
 };
 
 typedef std::tuple<int, int, int, int, int, int, int, int, int, uint32_t, int> TuneKey;
@@ -184,18 +200,23 @@ static bool kernel_supported(int kernel, const RegressArgs& a)
     if ((a.pb.flags & SR_LUMA_ONLY) && kernel != kKernelGeneral) return false;   // only the general kernel has the luma variant
     switch (kernel) {
     case kKernelSubset: return regress_subset_supported(a.mode, a.coef, a.coef_dtype, a.out, a.pb);
+    case kKernelListed: return regress_listed_supported(a.mode, a.coef, a.coef_dtype, a.idx, a.out, a.pb);
     case kKernelSecondLayout: return regress_tc_supported(a.mode, a.coef, a.coef_dtype, a.pb);
     case kKernelFirstLayout: return idx_vec_ok && umma_supported(a.mode, a.coef, a.coef_dtype, a.pb);
     default: return true;
     }
 }
 
-// The host rules: small global subsets on the FMA-pipe subset kernel; the second tensor-core layout for the other
+// The host rules: small global subsets on the FMA-pipe subset kernel; per-pixel lists with their values on the gather
+// kernel; the second tensor-core layout for the other
 // global subsets and for dense launches with few atoms; the first layout for the rest it supports; else the general kernel.
 static int default_kernel(const RegressArgs& a)
 {
+    const int forced = g_force_kernel.load(std::memory_order_relaxed);
+    if (forced >= 0 && kernel_supported(forced, a)) return forced;
     if (kernel_supported(kKernelSubset, a)) return kKernelSubset;
     const bool first = kernel_supported(kKernelFirstLayout, a), second = kernel_supported(kKernelSecondLayout, a);
+    if (kernel_supported(kKernelListed, a) && (!first || compact_prefers_listed(a.pb))) return kKernelListed;
     if (second && (a.mode == kModeGlobal || dense_prefers_second_layout(a.pb) || !first)) return kKernelSecondLayout;
     if (first) return kKernelFirstLayout;
     return kKernelGeneral;
@@ -205,6 +226,7 @@ static cudaError_t run_kernel(const TuneChoice& c, const RegressArgs& a)
 {
     switch (c.kernel) {
     case kKernelSubset: return launch_regress_subset(a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st, c.sub_th);
+    case kKernelListed: return launch_regress_listed(a.lr, a.coef, a.idx, a.dict, a.out, a.pb, a.st, c.sub_th);
     case kKernelSecondLayout: return launch_regress_tc(a.mode, a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st, c.tc);
     case kKernelFirstLayout: return launch_regress_umma(a.mode, a.lr, a.coef, a.idx, a.gamma, a.dict, a.out, a.pb, a.st);
     default: return launch_regress_fma(a.mode, a.lr, a.coef, a.coef_dtype, a.idx, a.gamma, a.dict, a.out, a.pb, a.st);
@@ -280,6 +302,11 @@ static int tune_shape(const RegressArgs& a, int reps, sr_tune_result* res)
         const int n = regress_subset_candidates(a.pb, ths, 8);
         for (int i = 0; i < n; ++i) { TuneChoice c; c.kernel = kKernelSubset; c.sub_th = ths[i]; cands.push_back(c); }
     }
+    if (kernel_supported(kKernelListed, a)) {
+        int ths[8];
+        const int n = regress_listed_candidates(a.pb, ths, 8);
+        for (int i = 0; i < n; ++i) { TuneChoice c; c.kernel = kKernelListed; c.sub_th = ths[i]; cands.push_back(c); }
+    }
     if (cands.empty()) { TuneChoice c; c.kernel = kKernelGeneral; cands.push_back(c); }
     cudaEvent_t e0, e1;
     if (cudaEventCreate(&e0) != cudaSuccess) return SR_ERR_CUDA;
@@ -304,7 +331,7 @@ static int tune_shape(const RegressArgs& a, int reps, sr_tune_result* res)
     }
     if (res) {
         res->kernel = pick.kernel;
-        res->tile_rows = pick.kernel == kKernelSecondLayout ? pick.tc.th : (pick.kernel == kKernelSubset ? pick.sub_th : 0);
+        res->tile_rows = pick.kernel == kKernelSecondLayout ? pick.tc.th : ((pick.kernel == kKernelSubset || pick.kernel == kKernelListed) ? pick.sub_th : 0);
         res->rows_per_step = pick.kernel == kKernelSecondLayout ? pick.tc.group : 0;
         res->candidates = (int32_t)cands.size();
         res->best_us = best_us;
@@ -562,6 +589,13 @@ int sr_test_lose_arrival(int launches)
 {
     if (launches < 0) return SR_ERR_SHAPE;
     g_lose_arrival.store(launches, std::memory_order_relaxed);
+    return SR_OK;
+}
+
+int sr_test_force_kernel(int kernel)
+{
+    if (kernel < -1 || kernel > kKernelListed) return SR_ERR_SHAPE;
+    g_force_kernel.store(kernel, std::memory_order_relaxed);
     return SR_OK;
 }
 

@@ -125,3 +125,5 @@ def test_wait_limit_is_returned_and_the_hook_validates_its_count(lib):
     assert sr.sr_set_wait_limit(old) == 12345
     assert lib.sr_test_lose_arrival(-1) == api.SR_ERR_SHAPE
     assert lib.sr_test_lose_arrival(0) == api.SR_OK
+    assert lib.sr_test_force_kernel(5) == api.SR_ERR_SHAPE and lib.sr_test_force_kernel(-2) == api.SR_ERR_SHAPE
+    assert lib.sr_test_force_kernel(-1) == api.SR_OK

@@ -24,12 +24,13 @@ def _calls():
     lr, dict_, coef = sr_inputs.make_inputs(wl)
     dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
     idx, sel = sr.sr_dict_select(dco, 8, want_sel=True)
+    idx16, sel16 = sr.sr_dict_select(dco, 16, want_sel=True)   # lists too long for the gather kernel (no waits) at this shape
     S = dev(np.arange(0, 72, 6, dtype=np.uint8))          # twelve atoms: more than the FMA-pipe subset kernel (no waits) takes
     return {
         "dense": lambda: sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5),
         "fused_select": lambda: sr.sr_dict_regress_selected(dlr, dco, None, None, ddi, 2, 5, 8),
         "index_planes": lambda: sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, 2, 5, 8),
-        "compact": lambda: sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, 2, 5, 8, sr.SR_COEF_COMPACT),
+        "compact": lambda: sr.sr_dict_regress_selected(dlr, sel16, idx16, None, ddi, 2, 5, 16, sr.SR_COEF_COMPACT),
         "global_subset": lambda: sr.sr_dict_regress_selected(dlr, dco, S, None, ddi, 2, 5, 12, sr.SR_IDX_GLOBAL),
         "dense_few_atoms": lambda: sr.sr_dict_regress_dense(dlr, dco[:, :16].contiguous(), ddi[:16].contiguous(), 2, 5),
     }
