@@ -127,16 +127,16 @@ static bool bad_out_flags(uint32_t flags, const sr_dims* d)
 static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 || (pb.k == 7 && pb.D <= 32); }
 
 // Which kernel takes a launch from index + value planes when both could. The gather kernel (sr_regress_listed.cu) pays
-// s * ceil(k^2 / 4) 16-byte shared-memory gathers per pixel and nothing per atom of the dictionary; the first
+// s * floor(k^2 / 4) 16-byte shared-memory gathers per pixel and nothing per atom of the dictionary; the first
 // tensor-core layout pays for clearing and filling a stage row of D coefficients per pixel and little per listed atom.
 // Measured on the 1080p sweep points and the 4K x2 batch (D = 16 / 32 / 72 / 128; k = 3 / 5 / 7; s = 4 / 8 / 16): the
-// gather kernel is 1.0 - 3.4 times faster wherever one of these holds, and up to two times slower at the far end
-// (k = 7, s = 16).
+// gather kernel is 1.0 - 3.7 times faster wherever this returns true, and up to 2.5 times slower at the far end
+// (k = 7, s = 16, few atoms). At scale 2 with 64 atoms or more the tensor-core layout has few stages left.
 static bool compact_prefers_listed(const Problem& pb)
 {
     const int gathers = pb.s * ((pb.k * pb.k + 3) / 4);
-    if (pb.D > 96 || gathers <= 28) return true;
-    if (pb.D >= 64) return gathers <= 52 || (gathers <= 56 && pb.r == 2);
+    if (pb.D > 96 || pb.k == 3 || gathers <= 28) return true;
+    if (pb.D >= 64) return gathers <= 52 || (pb.r == 2 && gathers <= 112);
     return false;
 }
 

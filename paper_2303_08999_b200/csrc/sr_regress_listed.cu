@@ -10,8 +10,10 @@
 // The gather sets the pace: every lane of a warp wants a different dictionary row, 16 bytes at a time. The dictionary
 // is therefore stored eight times, copy p in the 16-byte bank group p of every 128-byte line, and lane l reads copy
 // l % 8: the eight lanes that share a shared-memory cycle always hit eight different bank groups, whatever atoms they
-// ask for (D * ceil(k^2 / 4) * 128 bytes: 63 KB for 72 atoms of 5 x 5).
-// Bound: shared-memory bandwidth of the gather (s * ceil(k^2 / 4) * 16 bytes per pixel), then the fp32 pipe.
+// ask for. k^2 is odd: the last tap of every atom sits in a table of its own with one copy per lane (4-byte loads, lane
+// l reads bank l), so that no 16-byte gather is spent on a single tap (D * (floor(k^2 / 4) + 1) * 128 bytes: 63 KB for
+// 72 atoms of 5 x 5).
+// Bound: shared-memory bandwidth of the gather (s * (floor(k^2 / 4) * 16 + 4) bytes per pixel), then the fp32 pipe.
 //
 // One CTA of 512 threads per SM; its two halves of 256 threads walk different tiles (128 x th pixels, th = 8, 16 or
 // 24) with their own tile buffers and their own named barrier, so that one half builds its next up-sampled tile while
@@ -68,7 +70,8 @@ template <int K, int C, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __grid_constant__ ListedParams p)
 {
     constexpr int kk = K * K, P = (K - 1) / 2, UW = tile_uw(P), UW4 = UW / 4;
-    constexpr int NU = (kk + 3) / 4;              // 16-byte units of a dictionary row
+    constexpr int NU = kk / 4;                    // 16-byte units of a dictionary row: taps 0 .. 4 NU - 1; tap kk - 1 apart
+    static_assert(kk == 4 * NU + 1, "k^2 = 1 (mod 4) for odd k");
     constexpr int EP = K <= 5 ? 2 : 1;            // pixels whose filters are held at once (register budget)
     constexpr int NL = (K + 2) / 2;               // 8-byte loads that cover the K + 1 columns of a pixel pair's patches
     extern __shared__ __align__(16) float smem[];
@@ -79,22 +82,25 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
     const int tid = threadIdx.x, half = tid >> 8, ht = tid & (kHalfThreads - 1), warp = ht >> 5, lane = tid & 31;
     const int dict_units = pb.D * NU * 8;
     float4* sD = reinterpret_cast<float4*>(smem);                                      // [D][NU][8 copies]
-    float* hb = smem + 4 * dict_units + half * p.half_floats;
+    float* sT = smem + 4 * dict_units;                                                 // [D][32 copies]: last tap
+    const int last_floats = 32 * pb.D;
+    float* hb = sT + last_floats + half * p.half_floats;
     float* sU = hb;                                                                    // [C][uh][UW]
     float* sV = sU + C * g.uh * UW;                                                    // [C][uh][tcols]
     float* sL = sV + C * g.uh * g.tcols;                                               // [C * trows][tcols]
 
     // ---- set-up: tile buffers start as zeros (the up-sampling passes read a few values beyond the ones they weight)
     for (int i = tid; i < 2 * p.half_floats / 4; i += kThreads)
-        reinterpret_cast<float4*>(smem + 4 * dict_units)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4*>(sT + last_floats)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     fill_wpad(pb, wpad, tid, kThreads);
     for (int i = tid; i < dict_units; i += kThreads) {
         const int u = i >> 3, a = u / NU, j = u - a * NU;
         float v[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = 4 * j + e < kk ? __ldg(p.dict + (int64_t)a * kk + 4 * j + e) : 0.f;
+        for (int e = 0; e < 4; ++e) v[e] = __ldg(p.dict + (int64_t)a * kk + 4 * j + e);
         sD[i] = make_float4(v[0], v[1], v[2], v[3]);
     }
+    for (int i = tid; i < last_floats; i += kThreads) sT[i] = __ldg(p.dict + (int64_t)(i >> 5) * kk + kk - 1);
     __syncthreads();
 
     // this thread's part of the up-sampling passes of its half: a group of four columns and a row lane
@@ -106,6 +112,7 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
     const int bar_id = 1 + half;
     const int rsub = warp >> 1, pp = (warp & 1) * 32 + lane;      // row of a pass, pixel pair of the row
     const float4* my_dict = sD + (lane & 7);
+    const float* my_last = sT + lane;
 
     // lists of the 64 pixels this warp filters in row y of frame f: one 64-byte piece per index plane and one 128-byte
     // line per value plane, asked into L2 a row of work ahead
@@ -146,10 +153,13 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
             for (int e0 = 0; e0 < 2; e0 += EP) {
                 // ---- the filters of pixels e0 .. e0 + EP - 1: F[e][j] = taps 2 j, 2 j + 1
                 float2 F[EP][2 * NU];
+                float Fl[EP];                                // the last tap
 #pragma unroll
                 for (int e = 0; e < EP; ++e)
 #pragma unroll
                     for (int j = 0; j < 2 * NU; ++j) F[e][j] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int e = 0; e < EP; ++e) Fl[e] = 0.f;
                 for (int q0 = 0; q0 < p.natoms; q0 += 8) {
                     uint32_t iw[8], vw[8];
 #pragma unroll
@@ -175,8 +185,9 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
                                 for (int u = 0; u < NU; ++u) {
                                     const float4 d = dr[u * 8];
                                     F[e][2 * u] = __ffma2_rn(make_float2(d.x, d.y), vv, F[e][2 * u]);
-                                    if (4 * u + 2 < kk) F[e][2 * u + 1] = __ffma2_rn(make_float2(d.z, d.w), vv, F[e][2 * u + 1]);
+                                    F[e][2 * u + 1] = __ffma2_rn(make_float2(d.z, d.w), vv, F[e][2 * u + 1]);
                                 }
+                                Fl[e] = fmaf(my_last[a * 32], v, Fl[e]);
                             }
                         }
                     }
@@ -184,6 +195,9 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
                 // ---- applied to the up-sampled tile: pixel px, tap (a, b) reads row (row + a), column 2 pp + px + b
 #pragma unroll
                 for (int a = 0; a < K; ++a) {
+                    // keeps the compiler from hoisting every row's loads above the arithmetic (7 x 7: 21 rows of eight
+                    // values, which it then spills)
+                    asm volatile("" ::: "memory");
 #pragma unroll
                     for (int c = 0; c < C; ++c) {
                         const float2* up = reinterpret_cast<const float2*>(sU + (c * g.uh + row + a) * UW + 2 * pp);
@@ -200,7 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
 #pragma unroll
                             for (int b = 0; b < K; ++b) {
                                 const int tap = a * K + b;
-                                const float f = (tap & 1) ? F[e][tap >> 1].y : F[e][tap >> 1].x;
+                                const float f = tap == kk - 1 ? Fl[e] : ((tap & 1) ? F[e][tap >> 1].y : F[e][tap >> 1].x);
                                 acc[c][px] = fmaf(f, u[px + b], acc[c][px]);
                             }
                         }
@@ -249,7 +263,7 @@ size_t smem_for(const Problem& pb, int th, int& half_floats)
 {
     Geom g;
     half_floats = (int)((plan_geom(g, pb, th, nullptr) + 8 + 3) & ~(size_t)3);
-    const size_t dict = (size_t)pb.D * ((pb.k * pb.k + 3) / 4) * 128;
+    const size_t dict = (size_t)pb.D * (pb.k * pb.k / 4 + 1) * 128;     // the 16-byte units, eight copies each, and the last taps
     const size_t need = dict + 2 * (size_t)half_floats * 4;
     const DeviceInfo& di = device_info();
     return di.ok && need + kStaticReserve <= (size_t)di.smem_optin ? need : 0;

@@ -19,18 +19,26 @@ pytestmark = pytest.mark.gpu
 SHORT_BUDGET = 2_000_000   # SM cycles: about a millisecond
 
 
+def _on_kernel(kernel, fn):
+    sr.sr_test_force_kernel(kernel)
+    try:
+        return fn()
+    finally:
+        sr.sr_test_force_kernel(-1)
+
+
 def _calls():
     wl = sr_inputs.Workload("t", 1, 3, 24, 64, 2, D=72, k=5, coef_dtype="f16")
     lr, dict_, coef = sr_inputs.make_inputs(wl)
     dlr, dco, ddi = dev(lr), dev(coef), dev(dict_)
     idx, sel = sr.sr_dict_select(dco, 8, want_sel=True)
-    idx16, sel16 = sr.sr_dict_select(dco, 16, want_sel=True)   # lists too long for the gather kernel (no waits) at this shape
     S = dev(np.arange(0, 72, 6, dtype=np.uint8))          # twelve atoms: more than the FMA-pipe subset kernel (no waits) takes
     return {
         "dense": lambda: sr.sr_dict_regress_dense(dlr, dco, ddi, 2, 5),
         "fused_select": lambda: sr.sr_dict_regress_selected(dlr, dco, None, None, ddi, 2, 5, 8),
         "index_planes": lambda: sr.sr_dict_regress_selected(dlr, dco, idx, None, ddi, 2, 5, 8),
-        "compact": lambda: sr.sr_dict_regress_selected(dlr, sel16, idx16, None, ddi, 2, 5, 16, sr.SR_COEF_COMPACT),
+        # pinned to the first tensor-core layout: the host rules give this shape to the gather kernel, which has no waits
+        "compact": lambda: _on_kernel(1, lambda: sr.sr_dict_regress_selected(dlr, sel, idx, None, ddi, 2, 5, 8, sr.SR_COEF_COMPACT)),
         "global_subset": lambda: sr.sr_dict_regress_selected(dlr, dco, S, None, ddi, 2, 5, 12, sr.SR_IDX_GLOBAL),
         "dense_few_atoms": lambda: sr.sr_dict_regress_dense(dlr, dco[:, :16].contiguous(), ddi[:16].contiguous(), 2, 5),
     }
