@@ -25,7 +25,7 @@ Workloads: cfg1 (the default; cfg2 is the same frame) prints the one JSON line o
 coefficients, 128 x 128 output) and cfg3 (batch of four 4K frames) print one line of the same form. cfg4 is the shape
 sweep (LR 360 x 640, scale in {2,3,4}, D in {16,32,72,128}, k in {3,5,7}, s in {4,8,16}): one line per point and s, each
 with the per-path times and roofline fractions, the clocks seen during its timed region and the oracle timed on a
-small sample (`--points r3_D72_k5` restricts the sweep). Every path's roofline is the slowest of its bytes at the
+small sample (`--points r3_D72_k5` restricts the sweep, `--s 8` its list lengths). Every path's roofline is the slowest of its bytes at the
 measured HBM bandwidth, its selection-network operations at the measured integer max/min rate and its multiply-adds
 at the measured fp32 rate (both rates are measured at start-up by the library's probe kernels).
 `--workload producer` times the regression fused with the last layer of the coefficient network (sr_producer_regress, one
@@ -765,6 +765,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--points", default="", help="cfg4 only: comma-separated substrings of point names, e.g. r3_D72_k5")
+    ap.add_argument("--s", type=int, default=0, help="cfg4 only: keep one list length of the sweep's 4, 8, 16")
     ap.add_argument("--paths", default=",".join(PATHS), help="comma-separated subset of the step's paths (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -787,7 +788,7 @@ def main():
     elif sweep:
         want = [w for w in args.points.split(",") if w]
         wls = [replace(p, s=s) for p in sr_inputs.cfg4_points() for s in (4, 8, 16)
-               if s <= p.D and (not want or any(w in p.name for w in want))]
+               if s <= p.D and (not args.s or s == args.s) and (not want or any(w in p.name for w in want))]
     else:
         wls = [sr_inputs.CONFIGS[args.workload]]
     if args.impl == "reference":
