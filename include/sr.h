@@ -300,7 +300,8 @@ int sr_producer_regress(const float* lr, const void* feat, const void* folded, s
 /*
  * Sustained issue rate of an arithmetic pipe of the current device, for the roofline of the kernels that are bound by
  * one (the selection networks by integer max/min, the general and subset regressions by fp32 multiply-add):
- * kind 0 = integer max/min, kind 1 = fp32 multiply-add.  Runs a register-only kernel a few times on `stream`,
+ * kind 0 = integer max/min, kind 1 = fp32 multiply-add, kind 2 = packed fp32 multiply-add (fma.rn.f32x2, counted as two
+ * multiply-adds per lane and instruction).  Runs a register-only kernel a few times on `stream`,
  * synchronises it, and writes lane operations per second to *lane_ops_per_s (HOST pointer).  `scratch8` is 8 bytes of
  * device memory whose first int is read (any value) and which is otherwise left alone.  Introspection for benchmarks;
  * the paper has no counterpart.

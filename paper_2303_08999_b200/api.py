@@ -296,7 +296,8 @@ def sr_selection_search(G, b, hh, nrows: float, alpha: float, delta_alpha: float
 
 
 def sr_probe_rate(kind: int) -> float:
-    """Sustained lane operations per second of integer max/min (kind 0) or fp32 multiply-add (kind 1) on the current device."""
+    """Sustained lane operations per second of integer max/min (kind 0), fp32 multiply-add (kind 1) or packed fp32
+    multiply-add (kind 2, two per lane and instruction) on the current device."""
     scratch = torch.zeros(2, dtype=torch.int32, device="cuda")
     v = ctypes.c_double(0.0)
     _check(load_library().sr_probe_rate(kind, _ptr(scratch), ctypes.byref(v), _stream()), "sr_probe_rate")

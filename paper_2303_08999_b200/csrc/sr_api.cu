@@ -574,7 +574,7 @@ int sr_producer_regress(const float* lr, const void* feat, const void* folded, s
 int sr_probe_rate(int kind, void* scratch8, double* lane_ops_per_s, void* stream)
 {
     if (!scratch8 || !lane_ops_per_s) return SR_ERR_NULL;
-    if (kind != 0 && kind != 1) return SR_ERR_UNSUPPORTED;
+    if (kind < 0 || kind > 2) return SR_ERR_UNSUPPORTED;
     if (!aligned(scratch8, 4)) return SR_ERR_ALIGN;
     return probe_rate(kind, static_cast<int*>(scratch8), lane_ops_per_s, (cudaStream_t)stream) == cudaSuccess ? SR_OK : SR_ERR_CUDA;
 }

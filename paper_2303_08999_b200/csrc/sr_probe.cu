@@ -70,9 +70,30 @@ __global__ void __launch_bounds__(kThreads) probe_fma_kernel(const int* seed, fl
     if (acc == -1.f) sink[0] = acc;
 }
 
+// The packed form (fma.rn.f32x2: two multiply-adds per lane and instruction), same chains.
+__global__ void __launch_bounds__(kThreads) probe_fma2_kernel(const int* seed, float* sink)
+{
+    float2 a[kChains];
+    const float xs = 1.0f + 1e-7f * (float)(__ldg(seed) + threadIdx.x);
+    const float2 x = make_float2(xs, xs + 1e-7f), y = make_float2(1e-9f, 2e-9f);
+#pragma unroll
+    for (int i = 0; i < kChains; ++i) a[i] = make_float2((float)i, (float)(i + 1));
+#pragma unroll 1
+    for (int it = 0; it < kIters / 8; ++it) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int i = 0; i < kChains; ++i) a[i] = __ffma2_rn(a[i], x, y);
+    }
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < kChains; ++i) acc += a[i].x + a[i].y;
+    if (acc == -1.f) sink[0] = acc;
+}
+
 } // namespace
 
-// kind 0: integer max/min, kind 1: fp32 multiply-add. Lane operations per second; synchronises the stream.
+// kind 0: integer max/min, kind 1: fp32 multiply-add, kind 2: packed fp32 multiply-add (two per lane and instruction). Lane operations per second; synchronises the stream.
 cudaError_t probe_rate(int kind, int* scratch2 /* two ints of device memory */, double* lane_ops_per_s, cudaStream_t st)
 {
     const int ctas = sm_count() * 8;
@@ -85,7 +106,8 @@ cudaError_t probe_rate(int kind, int* scratch2 /* two ints of device memory */, 
     for (int rep = 0; rep < 4 && err == cudaSuccess; ++rep) {
         cudaEventRecord(e0, st);
         if (kind == 0) probe_minmax_kernel<<<ctas, kThreads, 0, st>>>(scratch2, scratch2 + 1);
-        else probe_fma_kernel<<<ctas, kThreads, 0, st>>>(scratch2, reinterpret_cast<float*>(scratch2 + 1));
+        else if (kind == 1) probe_fma_kernel<<<ctas, kThreads, 0, st>>>(scratch2, reinterpret_cast<float*>(scratch2 + 1));
+        else probe_fma2_kernel<<<ctas, kThreads, 0, st>>>(scratch2, reinterpret_cast<float*>(scratch2 + 1));
         count_launches(1);
         cudaEventRecord(e1, st);
         err = cudaEventSynchronize(e1);
@@ -97,7 +119,7 @@ cudaError_t probe_rate(int kind, int* scratch2 /* two ints of device memory */, 
     cudaEventDestroy(e1);
     if (err != cudaSuccess) return err;
     // max/min: (kIters / 8) trips x 2 passes x 2 sets x 38 operations per thread; multiply-add: kIters x kChains
-    const double per_thread = kind == 0 ? (double)(kIters / 8) * 2 * 2 * 38 : (double)kIters * kChains;
+    const double per_thread = kind == 0 ? (double)(kIters / 8) * 2 * 2 * 38 : (double)kIters * kChains * (kind == 2 ? 2 : 1);
     const double ops = (double)ctas * kThreads * per_thread;
     *lane_ops_per_s = ops / ((double)best_ms * 1e-3);
     return cudaSuccess;
