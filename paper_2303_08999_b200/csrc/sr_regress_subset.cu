@@ -91,17 +91,26 @@ __global__ void __launch_bounds__(kThreads, 2) regress_subset_kernel(const __gri
     const int h_lane = tid / UW4, h_cg = tid - h_lane * UW4, h_lanes = kThreads / UW4;
     const bool clamp01 = (pb.flags & SR_CLAMP01) != 0;
 
-    // the warp's work, in order: tile rows warp, warp + 8, ... of its CTA's tiles. (pf_t, pf_row) is the next row to
-    // fetch coefficients for; it always runs one row of work ahead of the row being computed.
-    int pf_t = blockIdx.x, pf_row = warp, buf = 0;
+    // The CTA's share of the image is a run of 8-row groups (the same number for every CTA to within one), cut into
+    // tiles of up to th rows. The warp's work, in order: tile rows warp, warp + 8, ... of its CTA's tiles. (pf_*) is the
+    // next row to fetch coefficients for; it always runs one row of work ahead of the row being computed.
+    const int run_end = run_bound(g, blockIdx.x + 1, gridDim.x);
+    int run_cur = run_bound(g, blockIdx.x, gridDim.x);
+    int pf_cur = run_cur, pf_rows = 0, pf_row = warp, buf = 0;
+    const __half* pf_src = nullptr;                          // this lane's four coefficients in row 0 of the tile, plane 0
+    auto pf_next_tile = [&]() {
+        int f, y0, x0;
+        if (!next_tile_of_run(g, pf_cur, run_end, f, y0, x0, pf_rows)) return false;
+        const int px = x0 + 4 * lane;
+        pf_src = px < pb.W ? p.coef + (int64_t)f * p.planes * plane_elems + (int64_t)y0 * pb.W + px : nullptr;
+        return true;
+    };
+    bool pf_tile = pf_next_tile();
     auto fetch_next = [&](int into) {
-        while (pf_t < g.num_tiles) {
-            int f, y0, x0, rows;
-            decode_tile(g, pf_t, f, y0, x0, rows);
-            if (pf_row < rows) {
-                const int px = x0 + 4 * lane;
-                if (px < pb.W) {
-                    const __half* src = p.coef + (int64_t)f * p.planes * plane_elems + (int64_t)(y0 + pf_row) * pb.W + px;
+        while (pf_tile) {
+            if (pf_row < pf_rows) {
+                if (pf_src) {
+                    const __half* src = pf_src + (int64_t)pf_row * pb.W;
 #pragma unroll
                     for (int q = 0; q < NQ; ++q)
                         if (q < p.natoms) cp_async_8(sPhi + (into * NQ + q) * kThreads + tid, src + plane_off[q]);
@@ -109,22 +118,36 @@ __global__ void __launch_bounds__(kThreads, 2) regress_subset_kernel(const __gri
                 pf_row += kWarps;
                 break;
             }
-            pf_t += gridDim.x;
+            pf_tile = pf_next_tile();
             pf_row = warp;
         }
         cp_async_commit();
     };
-    if ((int)blockIdx.x < g.num_tiles) prefetch_lr_window<P>(g, p.lr, blockIdx.x, sL, tid, kThreads);
+    {
+        int peek = run_cur;
+        LrWindow w0;
+        if (next_tile_of_run(g, peek, run_end, w0.f, w0.y0, w0.x0, w0.rows)) {
+            lr_window_of_tile<P>(g, w0);
+            prefetch_lr_window_of(g, p.lr, w0, sL, tid, kThreads);
+        }
+    }
     fetch_next(0);
-    for (int t = blockIdx.x; t < g.num_tiles; t += gridDim.x) {
-        LrWindow w;
-        lr_window<P>(g, t, w);
+    LrWindow w;
+    while (next_tile_of_run(g, run_cur, run_end, w.f, w.y0, w.x0, w.rows)) {
+        lr_window_of_tile<P>(g, w);
         const int uh = w.rows + 2 * P;
         cp_async_wait_all();
         __syncthreads();                                     // LR window landed; the previous tile's U is no longer read
         if (v_lane < v_lanes) vertical_pass(g, w, uh, P, sL, sV, v_i4, v_lane, v_lanes);
         __syncthreads();
-        if (t + (int)gridDim.x < g.num_tiles) prefetch_lr_window<P>(g, p.lr, t + gridDim.x, sL, tid, kThreads);
+        {
+            int peek = run_cur;
+            LrWindow wn;
+            if (next_tile_of_run(g, peek, run_end, wn.f, wn.y0, wn.x0, wn.rows)) {
+                lr_window_of_tile<P>(g, wn);
+                prefetch_lr_window_of(g, p.lr, wn, sL, tid, kThreads);
+            }
+        }
         if (h_lane < h_lanes) horizontal_pass<P>(g, wpad, w, uh, sV, sU, h_cg, h_lane, h_lanes);
         __syncthreads();                                     // the U tile is complete
 
@@ -229,11 +252,10 @@ const DeviceInfo& device_info()
 constexpr int kStaticReserve = 2048;   // static shared memory + the per-CTA system reservation
 
 
-// Tile height: the tiles are dealt round-robin to the resident CTAs, a warp takes every eighth row of a tile, so a
-// tile costs ceil(th / 8) row passes plus its up-sampled tile (th + k - 1 rows) and three CTA-wide barriers; the
-// launch takes as long as the CTA with the most tiles. Units: warp instructions. The per-tile term is set from
-// timings (1080p x4, s = 8: 59 / 58 / 51 us at th = 8 / 16 / 24): the tallest tile wins although it divides the
-// frame less evenly, because a tile's fixed work is about as long as sixteen rows of filtering.
+// Tile height: every resident CTA gets the same run of 8-row groups (to within one) and cuts it into tiles of up to th
+// rows; a warp takes every eighth row of a tile, so a run costs one row pass per group plus, per tile, its up-sampled
+// tile (th + k - 1 rows) and three CTA-wide barriers. Units: warp instructions. The per-tile term is set from timings
+// (1080p x4, s = 8): a tile's fixed work is about as long as sixteen rows of filtering, so the tallest tile wins.
 int choose_th(const Problem& pb, int nq, size_t& smem_bytes, int& ctas, int g_forced_th = 0)
 {
     const DeviceInfo& di = device_info();
@@ -246,11 +268,14 @@ int choose_th(const Problem& pb, int nq, size_t& smem_bytes, int& ctas, int g_fo
         Geom g;
         const size_t floats = ((plan_geom(g, pb, th, nullptr) + 2 * pb.k * pb.k * nq + 8 + 3) & ~(size_t)3) + 2 * nq * kThreads * 2;
         if (floats * 4 > (size_t)per_cta) continue;
-        const long long tiles = (long long)g.num_tiles;
-        const int c = tiles < 2LL * di.sms ? (int)tiles : 2 * di.sms;
-        const long long waves = (tiles + c - 1) / c;
+        const long long groups = (long long)g.num_groups;
+        const int c = groups < 2LL * di.sms ? (int)groups : 2 * di.sms;
+        // a CTA's run of ceil(groups / c) 8-row groups costs its row passes plus one up-sampled tile (th + k - 1 rows
+        // and three CTA-wide barriers) per th rows
+        const long long per_cta = (groups + c - 1) / c;
+        const long long tiles = (per_cta * 8 + th - 1) / th;
         const double row_pass = 8.0 * (nq * pb.k * pb.k * 0.625 + pb.c * pb.k * pb.k * 4 + 80);
-        const double cost = (double)waves * ((th / 8 + 2) * row_pass + g.uh * 175.0);
+        const double cost = (double)per_cta * row_pass + (double)tiles * (2 * row_pass + g.uh * 175.0);
         if (best_th == 0 || cost < best) { best_th = th; best = cost; smem_bytes = floats * 4; ctas = c; }
     }
     (void)tiles_x;

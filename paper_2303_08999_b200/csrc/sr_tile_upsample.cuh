@@ -26,6 +26,7 @@ struct Geom {
     uint32_t r_magic;     // ceil(2^32 / r): floor(x / r) == umulhi(x, r_magic) for 0 <= x < 2^29 (r >= 2)
     uint32_t tc4_magic;   // same for tcols / 4
     int tiles_x, tiles_y, num_tiles;
+    int gps, num_groups;  // 8-row groups per column strip (ceil(H / 8)) and in all strips of all frames
 };
 
 // U tile width for patch radius P: tile + halo, rounded up to 4 for 16-byte rows.
@@ -48,6 +49,8 @@ inline size_t plan_geom(Geom& g, const Problem& pb, int th, const float* lr, int
     g.tiles_x = (pb.W + tw - 1) / tw;
     g.tiles_y = (pb.H + th - 1) / th;
     g.num_tiles = g.tiles_x * g.tiles_y * pb.n;
+    g.gps = (pb.H + 7) / 8;
+    g.num_groups = g.gps * g.tiles_x * pb.n;
     return (size_t)pb.c * g.uh * UW + (size_t)pb.c * g.uh * g.tcols + (size_t)pb.c * g.trows * g.tcols;
 }
 
@@ -66,6 +69,28 @@ __device__ __forceinline__ void decode_tile(const Geom& p, int t, int& f, int& y
     rows = min(p.th, p.pb.H - y0);
 }
 
+// A worker's share of the image as a run of consecutive 8-row groups [cur, end) of the flattened space
+// [frame][column strip][group of 8 rows]: worker j of nworkers takes [j T / nworkers, (j + 1) T / nworkers), T =
+// num_groups, so that every worker filters the same number of rows to within one group, whatever the frame height.
+// next_tile_of_run cuts the next tile off the run: up to th rows (th a multiple of 8), never across a strip's end.
+__device__ __forceinline__ int run_bound(const Geom& p, int j, int nworkers)
+{
+    return (int)(((long long)j * p.num_groups) / nworkers);
+}
+
+__device__ __forceinline__ bool next_tile_of_run(const Geom& p, int& cur, int end, int& f, int& y0, int& x0, int& rows)
+{
+    if (cur >= end) return false;
+    const int strip = cur / p.gps, gy = cur - strip * p.gps;
+    const int ng = min(min(p.th >> 3, p.gps - gy), end - cur);
+    f = strip / p.tiles_x;
+    x0 = (strip - f * p.tiles_x) * p.tw;
+    y0 = gy * 8;
+    rows = min(ng * 8, p.pb.H - y0);
+    cur += ng;
+    return true;
+}
+
 // LR pixels a tile (plus patch halo) needs for its taps: rows lr_lo .. lr_lo + nrows - 1 and columns
 // col_a .. col_a + 4 nc4 - 1 (col_a a multiple of 4, possibly negative; reads clamp to the image).
 struct LrWindow { int f, y0, x0, rows, lr_lo, nrows, col_a, nc4; };
@@ -78,12 +103,12 @@ __device__ __forceinline__ int first_tap(const Geom& p, int Z, int& phase)
     return q + p.pb.ph.base[phase];
 }
 
+// Fills the window fields of g from its tile fields (f, y0, x0, rows).
 template <int P, int TWD = TW>
-__device__ __forceinline__ void lr_window(const Geom& p, int t, LrWindow& g)
+__device__ __forceinline__ void lr_window_of_tile(const Geom& p, LrWindow& g)
 {
     constexpr int UW = tile_uw(P, TWD);
     const Problem& pb = p.pb;
-    decode_tile(p, t, g.f, g.y0, g.x0, g.rows);
     int ph;
     g.lr_lo = first_tap(p, clampi(g.y0 - P, 0, pb.H - 1), ph);
     g.nrows = first_tap(p, clampi(g.y0 + g.rows - 1 + P, 0, pb.H - 1), ph) + 3 - g.lr_lo + 1;      // <= trows
@@ -91,6 +116,13 @@ __device__ __forceinline__ void lr_window(const Geom& p, int t, LrWindow& g)
     const int col_hi = first_tap(p, clampi(g.x0 - P + UW - 1, 0, pb.W - 1), ph) + 3;
     g.col_a = col_lo & ~3;                                       // rounds down, also for negative values
     g.nc4 = (col_hi - g.col_a) / 4 + 1;                          // <= tcols / 4
+}
+
+template <int P, int TWD = TW>
+__device__ __forceinline__ void lr_window(const Geom& p, int t, LrWindow& g)
+{
+    decode_tile(p, t, g.f, g.y0, g.x0, g.rows);
+    lr_window_of_tile<P, TWD>(p, g);
 }
 
 __device__ __forceinline__ void cp_async_4(float* dst_smem, const float* src)
@@ -105,13 +137,10 @@ __device__ __forceinline__ void cp_async_16(float* dst_smem, const float* src)
 // Fetches the LR window of tile t into dstL with asynchronous copies: 16 bytes where the four columns lie inside the
 // image and the row is aligned, single clamped elements at the borders. Thread `me` of `nthr`; the caller waits for
 // the copies (cp.async.wait_all or an mbarrier arrival).
-template <int P, int TWD = TW>
-__device__ __forceinline__ void prefetch_lr_window(const Geom& p, const float* lr, int t, float* dstL, int me, int nthr)
+__device__ __forceinline__ void prefetch_lr_window_of(const Geom& p, const float* lr, const LrWindow& g, float* dstL, int me, int nthr)
 {
     const Problem& pb = p.pb;
     const int C = pb.c;
-    LrWindow g;
-    lr_window<P, TWD>(p, t, g);
     const int tc4 = p.tcols >> 2;
     const int total = C * g.nrows * tc4;
     for (int e = me; e < total; e += nthr) {
@@ -130,6 +159,14 @@ __device__ __forceinline__ void prefetch_lr_window(const Geom& p, const float* l
             }
         }
     }
+}
+
+template <int P, int TWD = TW>
+__device__ __forceinline__ void prefetch_lr_window(const Geom& p, const float* lr, int t, float* dstL, int me, int nthr)
+{
+    LrWindow g;
+    lr_window<P, TWD>(p, t, g);
+    prefetch_lr_window_of(p, lr, g, dstL, me, nthr);
 }
 
 // Vertical pass on the LR columns of the window: V[ch][uy][i] = sum_a wy[a] * L[ch][first tap of row uy + a][i], four
