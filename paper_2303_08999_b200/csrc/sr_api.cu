@@ -129,15 +129,15 @@ static bool dense_prefers_second_layout(const Problem& pb) { return pb.D <= 16 |
 // Which kernel takes a launch from index + value planes when both could. The gather kernel (sr_regress_listed.cu) pays
 // s * floor(k^2 / 4) 16-byte shared-memory gathers per pixel and nothing per atom of the dictionary; the first
 // tensor-core layout pays for clearing and filling a stage row of D coefficients per pixel and little per listed atom.
-// Measured on the 1080p sweep points and the 4K x2 batch (D = 16 / 32 / 72 / 128; k = 3 / 5 / 7; s = 4 / 8 / 16): the
-// gather kernel is 1.0 - 3.7 times faster wherever this returns true, and up to 2.5 times slower at the far end
-// (k = 7, s = 16, few atoms). At scale 2 with 64 atoms or more the tensor-core layout has few stages left.
+// Measured on the 1080p sweep points and the 4K x2 batch (D = 16 / 32 / 72 / 128; k = 3 / 5 / 7; s = 4 / 8 / 16), both
+// kernels forced in turn: the gather kernel is 1.0 - 3.7 times faster wherever this returns true, and up to two times
+// slower at the far end (k = 7, s = 16, few atoms).
 static bool compact_prefers_listed(const Problem& pb)
 {
-    const int gathers = pb.s * ((pb.k * pb.k + 3) / 4);
-    if (pb.D > 96 || pb.k == 3 || gathers <= 28) return true;
-    if (pb.D >= 64) return gathers <= 52 || (pb.r == 2 && gathers <= 112);
-    return false;
+    const int gathers = pb.s * ((pb.k * pb.k + 3) / 4);      // 16-byte units of dictionary per pixel
+    if (pb.D > 96 || gathers <= 52) return true;
+    if (pb.D >= 64) return gathers <= 104 || (pb.r == 2 && gathers <= 112);
+    return pb.r == 2 && gathers <= 56;
 }
 
 // ---- which kernel runs a regression, and in which launch shape ----------------------------------------------------------

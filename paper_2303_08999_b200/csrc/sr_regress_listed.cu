@@ -124,18 +124,35 @@ __global__ void __launch_bounds__(kThreads, 1) regress_listed_kernel(const __gri
         }
     };
 
-    const int t0 = 2 * blockIdx.x + half, tstride = 2 * gridDim.x;
-    if (t0 < g.num_tiles) prefetch_lr_window<P>(g, p.lr, t0, sL, ht, kHalfThreads);
-    for (int t = t0; t < g.num_tiles; t += tstride) {
-        LrWindow w;
-        lr_window<P>(g, t, w);
+    // A half's share of the image is a run of 8-row groups (the same number for every half to within one), cut into
+    // tiles of up to th rows.
+    const int run_end = run_bound(g, 2 * blockIdx.x + half + 1, 2 * gridDim.x);
+    int run_cur = run_bound(g, 2 * blockIdx.x + half, 2 * gridDim.x);
+    {
+        int peek = run_cur;
+        LrWindow w0;
+        if (next_tile_of_run(g, peek, run_end, w0.f, w0.y0, w0.x0, w0.rows)) {
+            lr_window_of_tile<P>(g, w0);
+            prefetch_lr_window_of(g, p.lr, w0, sL, ht, kHalfThreads);
+        }
+    }
+    LrWindow w;
+    while (next_tile_of_run(g, run_cur, run_end, w.f, w.y0, w.x0, w.rows)) {
+        lr_window_of_tile<P>(g, w);
         const int uh = w.rows + 2 * P;
         prefetch_lists(w.f, w.y0 + rsub, w.x0 + 64 * (warp & 1));
         cp_async_wait_all();
         bar_sync(bar_id, kHalfThreads);                      // LR window landed; the previous tile's U is no longer read
         if (v_lane < v_lanes) vertical_pass(g, w, uh, P, sL, sV, v_i4, v_lane, v_lanes);
         bar_sync(bar_id, kHalfThreads);
-        if (t + tstride < g.num_tiles) prefetch_lr_window<P>(g, p.lr, t + tstride, sL, ht, kHalfThreads);
+        {
+            int peek = run_cur;
+            LrWindow wn;
+            if (next_tile_of_run(g, peek, run_end, wn.f, wn.y0, wn.x0, wn.rows)) {
+                lr_window_of_tile<P>(g, wn);
+                prefetch_lr_window_of(g, p.lr, wn, sL, ht, kHalfThreads);
+            }
+        }
         if (h_lane < h_lanes) horizontal_pass<P>(g, wpad, w, uh, sV, sU, h_cg, h_lane, h_lanes);
         bar_sync(bar_id, kHalfThreads);                      // the U tile is complete
 
@@ -269,8 +286,8 @@ size_t smem_for(const Problem& pb, int th, int& half_floats)
     return di.ok && need + kStaticReserve <= (size_t)di.smem_optin ? need : 0;
 }
 
-// Tile height: the tiles are dealt round-robin to the 2 x CTAs halves and the launch takes as long as the half with the
-// most tiles; a tile costs its rows (in passes of four) plus its up-sampled tile of th + k - 1 rows. Units: row passes.
+// Tile height: every half gets the same run of 8-row groups (to within one) and cuts it into tiles of up to th rows; a
+// run costs its rows (in passes of four) plus, per tile, an up-sampled tile of th + k - 1 rows. Units: row passes.
 Plan choose_plan(const Problem& pb, int th_forced)
 {
     Plan best;
@@ -284,10 +301,11 @@ Plan choose_plan(const Problem& pb, int th_forced)
         if (smem == 0) continue;
         Geom g;
         plan_geom(g, pb, th, nullptr);
-        const long long tiles = g.num_tiles;
-        const long long halves = tiles < 2LL * di.sms ? tiles : 2LL * di.sms;
-        const long long waves = (tiles + halves - 1) / halves;
-        const double cost = (double)waves * (th / kRowsPerPass + 0.12 * g.uh);
+        const long long groups = g.num_groups;
+        const long long halves = groups < 2LL * di.sms ? groups : 2LL * di.sms;
+        const long long per_half = (groups + halves - 1) / halves;               // 8-row groups in a half's run
+        const long long tiles = (per_half * 8 + th - 1) / th;
+        const double cost = (double)per_half * (8 / kRowsPerPass) + (double)tiles * 0.12 * g.uh;
         if (best.th == 0 || cost < best_cost) {
             best.th = th; best.smem = smem; best.half_floats = hf; best.ctas = (int)((halves + 1) / 2);
             best_cost = cost;
