@@ -9,7 +9,7 @@
 //   bitonic sequence holding the S best of both), bitonic-merge it back to sorted order (S/2 * log2 S exchanges).
 // Per pixel and plane that is about 8.75 min/max for S = 8 (630 per pixel at D = 72) against 16 for plain insertion.
 // The kernel is bound by the integer ALU rate or by HBM, whichever is slower for the shape.
-// With 16-byte aligned planes the block first stages its 512 pixels x D planes in shared memory (select_tile_kernel)
+// With 16-byte aligned planes the block first stages its 256 pixels x D planes in shared memory (select_tilef_kernel)
 // and the threads read their words, and at the end the selected values, from there.
 #include "sr_common.cuh"
 
@@ -150,13 +150,16 @@ select_pair_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, _
     }
 }
 
-// Same selection with the block's coefficients staged in shared memory first: a block owns 512 consecutive pixels
-// of a frame, copies their D planes with 16-byte asynchronous copies ([D][512] binary16), and every thread then reads
+// Same selection with the block's coefficients staged in shared memory first: a block owns TP = 256 consecutive pixels
+// of a frame, copies their D planes with 16-byte asynchronous copies ([D][TP] binary16), and every thread then reads
 // its pixel pair's words from there. The selected values are picked out of the same tile at the end, so no
 // coefficient is fetched from global memory twice (on frames whose planes are many megabytes apart the re-read of
 // the selected values used to miss the L2 and cost half as much again as the selection itself).
-// Needs 16-byte aligned planes (H * W a multiple of 8) and D KiB of shared memory.
-constexpr int kSelTilePixels = 512;
+// Needs 16-byte aligned planes (H * W a multiple of 8) and D / 2 KiB of shared memory. Shared memory, not registers,
+// limits the resident pixels (2 D bytes each: about 1500 per SM at D = 72 whatever the tile size); the smaller tile
+// gives more, shorter load and compute phases to interleave (six blocks per SM instead of three: 3 % faster at s = 8,
+// 8 % at s = 16 on the 1080p frame).
+constexpr int kSelTilePixels = 256;
 
 // Byte permute with the full selector: bit 3 of a selector nibble replicates the sign bit of the selected byte instead
 // of copying it (the intrinsic only documents the low three bits).
@@ -275,116 +278,31 @@ template <int S> __device__ __forceinline__ void merge_top_f(float* top, const f
 
 constexpr float kKeyMagic = 8388608.f;   // 2^23: the bits 0x4B000000 | key are the fp32 number 2^23 + key
 
-template <int S>
-__global__ void __launch_bounds__(256)
-select_tile_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
-                   const __grid_constant__ Problem pb, int tiles_per_frame)
-{
-    extern __shared__ __align__(16) uint8_t tile[];          // [D][512] binary16
-    const int64_t HW = (int64_t)pb.H * pb.W;
-    const int D = pb.D, s = pb.s, tid = threadIdx.x;
-    const int64_t f = blockIdx.x / tiles_per_frame;
-    const int64_t p0 = (int64_t)(blockIdx.x - f * tiles_per_frame) * kSelTilePixels;   // first pixel of the tile
-    const __half* cp = coef + f * D * HW + p0;
-    {
-        const uint32_t tile_s = (uint32_t)__cvta_generic_to_shared(tile);
-        const int chunk = tid & 63;                          // 16-byte chunk (8 pixels) of a plane's 1 KiB row
-        const uint32_t bytes = p0 + chunk * 8 < HW ? 16u : 0u;   // chunks beyond the frame are zero-filled
-        const __half* src = cp + (bytes ? chunk * 8 : 0);
-        for (int l = tid >> 6; l < D; l += 4)
-            sel_cp_async_16(tile_s + (uint32_t)l * 1024u + (uint32_t)chunk * 16u, src + (int64_t)l * HW, bytes);
-        asm volatile("cp.async.wait_all;" ::: "memory");
-    }
-    __syncthreads();
-    const int64_t pix = p0 + 2 * tid;
-    if (pix >= HW) return;
-    const uint32_t* wp = reinterpret_cast<const uint32_t*>(tile) + tid;   // + 256 words per plane
-    int ta[S], tb[S];
-#pragma unroll
-    for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1;
-    int l0 = 0;
-    // Tags of four planes per register: byte j of tags[q] = 255 - (l0 + 4 q + j). A group moves them all down by S with
-    // one subtraction per register (no byte ever borrows: a tag is at least 255 - 199), instead of one per key.
-    uint32_t tags[S / 4];
-#pragma unroll
-    for (int q = 0; q < S / 4; ++q)
-        tags[q] = (255u - 4u * q) | ((254u - 4u * q) << 8) | ((253u - 4u * q) << 16) | ((252u - 4u * q) << 24);
-    for (; l0 + S <= D; l0 += S) {                           // whole groups: no per-key guards
-        uint32_t w[S];
-#pragma unroll
-        for (int i = 0; i < S; ++i) w[i] = wp[(l0 + i) * 256];
-        int ga[S], gb[S];
-#pragma unroll
-        for (int i = 0; i < S; ++i) {
-            // key = (tag, magnitude low byte, magnitude high byte, 0): one byte permute per pixel out of (signs cleared,
-            // four tags); the top byte replicates the (cleared) sign bit of a magnitude byte, i.e. zero
-            const uint32_t m2 = w[i] & 0x7FFF7FFFu;
-            ga[i] = (int)prmt(m2, tags[i >> 2], 0x9100u | (uint32_t)(4 + (i & 3)));
-            gb[i] = (int)prmt(m2, tags[i >> 2], 0x9320u | (uint32_t)(4 + (i & 3)));
-        }
-        sort_desc<S>(ga);
-        sort_desc<S>(gb);
-        merge_top<S>(ta, ga);
-        merge_top<S>(tb, gb);
-#pragma unroll
-        for (int q = 0; q < S / 4; ++q) tags[q] -= 0x01010101u * (uint32_t)S;
-    }
-    if (l0 < D) {                                            // last, partial group
-        int ga[S], gb[S];
-#pragma unroll
-        for (int i = 0; i < S; ++i) {
-            ga[i] = gb[i] = -1;
-            if (l0 + i < D) {
-                const uint32_t tag = (uint32_t)(255 - (l0 + i)), m2 = wp[(l0 + i) * 256] & 0x7FFF7FFFu;
-                ga[i] = (int)__byte_perm(m2, tag, 0x5104);
-                gb[i] = (int)__byte_perm(m2, tag, 0x5324);
-            }
-        }
-        sort_desc<S>(ga);
-        sort_desc<S>(gb);
-        merge_top<S>(ta, ga);
-        merge_top<S>(tb, gb);
-    }
-    const __half* th = reinterpret_cast<const __half*>(tile) + 2 * tid;
-#pragma unroll
-    for (int q = 0; q < S; ++q) {
-        if (q < s) {
-            const int a = 255 - (ta[q] & 255), b = 255 - (tb[q] & 255);
-            const int64_t o = (f * s + q) * HW + pix;
-            *reinterpret_cast<uchar2*>(idx + o) = make_uchar2((unsigned char)a, (unsigned char)b);
-            if (sel) *reinterpret_cast<__half2*>(sel + o) = __halves2half2(th[a * kSelTilePixels], th[b * kSelTilePixels + 1]);
-        }
-    }
-}
-
-// The same tile kernel with the keys held as fp32 numbers, so that part of the compare-exchanges run
-// on the FMA pipe (see cxf). Three tags and the exponent byte 0x4B share a register: one prmt builds the bits of
-// 2^23 + key, one subtraction (FMA pipe) leaves the key.
-template <int S>
-__global__ void __launch_bounds__(256)
+template <int S, int TP>   // TP: pixels per tile (512 or 256), two per thread
+__global__ void __launch_bounds__(TP / 2)
 select_tilef_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, __half* __restrict__ sel,
                     const __grid_constant__ Problem pb, int tiles_per_frame)
 {
     constexpr int NT = (S + 2) / 3;                          // tag registers: three tags each
-    extern __shared__ __align__(16) uint8_t tile[];          // [D][512] binary16
+    extern __shared__ __align__(16) uint8_t tile[];          // [D][TP] binary16
     const int64_t HW = (int64_t)pb.H * pb.W;
     const int D = pb.D, s = pb.s, tid = threadIdx.x;
     const int64_t f = blockIdx.x / tiles_per_frame;
-    const int64_t p0 = (int64_t)(blockIdx.x - f * tiles_per_frame) * kSelTilePixels;   // first pixel of the tile
+    const int64_t p0 = (int64_t)(blockIdx.x - f * tiles_per_frame) * TP;   // first pixel of the tile
     const __half* cp = coef + f * D * HW + p0;
     {
         const uint32_t tile_s = (uint32_t)__cvta_generic_to_shared(tile);
-        const int chunk = tid & 63;                          // 16-byte chunk (8 pixels) of a plane's 1 KiB row
+        const int chunk = tid & (TP / 8 - 1);                // 16-byte chunk (8 pixels) of a plane's row of TP pixels
         const uint32_t bytes = p0 + chunk * 8 < HW ? 16u : 0u;   // chunks beyond the frame are zero-filled
         const __half* src = cp + (bytes ? chunk * 8 : 0);
-        for (int l = tid >> 6; l < D; l += 4)
-            sel_cp_async_16(tile_s + (uint32_t)l * 1024u + (uint32_t)chunk * 16u, src + (int64_t)l * HW, bytes);
+        for (int l = tid / (TP / 8); l < D; l += 4)
+            sel_cp_async_16(tile_s + (uint32_t)l * (uint32_t)(2 * TP) + (uint32_t)chunk * 16u, src + (int64_t)l * HW, bytes);
         asm volatile("cp.async.wait_all;" ::: "memory");
     }
     __syncthreads();
     const int64_t pix = p0 + 2 * tid;
     if (pix >= HW) return;
-    const uint32_t* wp = reinterpret_cast<const uint32_t*>(tile) + tid;   // + 256 words per plane
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(tile) + tid;   // + TP / 2 words per plane
     float ta[S], tb[S];
 #pragma unroll
     for (int i = 0; i < S; ++i) ta[i] = tb[i] = -1.f;
@@ -397,7 +315,7 @@ select_tilef_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, 
     for (; l0 + S <= D; l0 += S) {                           // whole groups: no per-key guards
         uint32_t w[S];
 #pragma unroll
-        for (int i = 0; i < S; ++i) w[i] = wp[(l0 + i) * 256];
+        for (int i = 0; i < S; ++i) w[i] = wp[(l0 + i) * (TP / 2)];
         float ga[S], gb[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) {
@@ -419,7 +337,7 @@ select_tilef_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, 
         for (int i = 0; i < S; ++i) {
             ga[i] = gb[i] = -1.f;
             if (l0 + i < D) {
-                const uint32_t m2 = wp[(l0 + i) * 256] & 0x7FFF7FFFu;
+                const uint32_t m2 = wp[(l0 + i) * (TP / 2)] & 0x7FFF7FFFu;
                 ga[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7100u | (uint32_t)(4 + i % 3))) - kKeyMagic;
                 gb[i] = __uint_as_float(prmt(m2, tags[i / 3], 0x7320u | (uint32_t)(4 + i % 3))) - kKeyMagic;
             }
@@ -436,7 +354,7 @@ select_tilef_kernel(const __half* __restrict__ coef, uint8_t* __restrict__ idx, 
             const int a = 255 - (int)(__float_as_uint(ta[q] + kKeyMagic) & 255u), b = 255 - (int)(__float_as_uint(tb[q] + kKeyMagic) & 255u);
             const int64_t o = (f * s + q) * HW + pix;
             *reinterpret_cast<uchar2*>(idx + o) = make_uchar2((unsigned char)a, (unsigned char)b);
-            if (sel) *reinterpret_cast<__half2*>(sel + o) = __halves2half2(th[a * kSelTilePixels], th[b * kSelTilePixels + 1]);
+            if (sel) *reinterpret_cast<__half2*>(sel + o) = __halves2half2(th[a * TP], th[b * TP + 1]);
         }
     }
 }
@@ -537,21 +455,22 @@ bool tile_path_ok(const void* coef, const Problem& pb)
            (HW + kSelTilePixels - 1) / kSelTilePixels * pb.n <= 0x7FFFFFFF;
 }
 
-template <int S, bool FLOAT_KEYS = false>
-cudaError_t launch_tile_s(const __half* c, uint8_t* idx, __half* sl, const Problem& pb, cudaStream_t st)
+template <int S, int TP>
+cudaError_t launch_tilef_s(const __half* c, uint8_t* idx, __half* sl, const Problem& pb, cudaStream_t st)
 {
-    const size_t smem = (size_t)pb.D * kSelTilePixels * sizeof(__half);
-    auto kern = FLOAT_KEYS ? select_tilef_kernel<S> : select_tile_kernel<S>;
+    const size_t smem = (size_t)pb.D * TP * sizeof(__half);
+    auto kern = select_tilef_kernel<S, TP>;
     static bool configured[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * kSelTilePixels * (int)sizeof(__half));
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * TP * (int)sizeof(__half));
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    const int tiles_per_frame = (int)(((int64_t)pb.H * pb.W + kSelTilePixels - 1) / kSelTilePixels);
-    kern<<<(unsigned)(tiles_per_frame * pb.n), 256, smem, st>>>(c, idx, sl, pb, tiles_per_frame);
+    const int64_t tiles_per_frame = ((int64_t)pb.H * pb.W + TP - 1) / TP;
+    if (tiles_per_frame * pb.n > 0x7FFFFFFF) return cudaErrorInvalidConfiguration;
+    kern<<<(unsigned)(tiles_per_frame * pb.n), TP / 2, smem, st>>>(c, idx, sl, pb, (int)tiles_per_frame);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -560,9 +479,9 @@ cudaError_t launch_tile(const void* coef, uint8_t* idx, void* sel, const Problem
 {
     const __half* c = (const __half*)coef;
     __half* sl = (__half*)sel;
-    if (pb.s <= 4) return launch_tile_s<4, true>(c, idx, sl, pb, st);
-    if (pb.s <= 8) return launch_tile_s<8, true>(c, idx, sl, pb, st);
-    return launch_tile_s<16, true>(c, idx, sl, pb, st);
+    if (pb.s <= 4) return launch_tilef_s<4, kSelTilePixels>(c, idx, sl, pb, st);
+    if (pb.s <= 8) return launch_tilef_s<8, kSelTilePixels>(c, idx, sl, pb, st);
+    return launch_tilef_s<16, kSelTilePixels>(c, idx, sl, pb, st);
 }
 
 cudaError_t launch_pair(const void* coef, uint8_t* idx, void* sel, const Problem& pb, cudaStream_t st)
