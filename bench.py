@@ -97,9 +97,9 @@ def load_peaks():
 
 
 # DRAM bytes per HR pixel seen by ncu (dram__bytes_read.sum + dram__bytes_write.sum) for each path's kernel on the
-# 1080p x4 frame (cfg1 / cfg2 only; figures and commands are in profiles/). None = not captured. The global-subset
-# figure is below its algorithmic bytes because the output frame (24.9 MB) is still in the 126 MB L2 when the kernel ends.
-NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": None, "dense": 154.2, "select": 161.7, "compact": 25.5, "fused": 154.3, "global": 17.1}
+# 1080p x4 frame (cfg1 / cfg2 only; figures and commands are in profiles/dram_traffic_cfg1.md). Figures below a path's
+# algorithmic bytes: the output (24.9 MB frame, 49.8 MB of index + value planes) is still in the 126 MB L2 when the kernel ends.
+NCU_TRAFFIC_BYTES_PER_PIXEL = {"bicubic": 0.8, "dense": 154.2, "select": 163.5, "compact": 25.5, "fused": 154.1, "global": 16.8}
 
 
 def selection_network_ops_per_pixel(path: str, D: int, s: int):
